@@ -1,0 +1,139 @@
+/*
+ * atflash.h - C ABI of the B200 (sm_100a) library for causal GQA attention with
+ * per-RoPE-wavelength distance windows.
+ *
+ * The score of query position n against key position m (distance z = n - m >= 0) is the sum
+ * over RoPE frequency pairs r of the pair's contribution (paper Eq. 1); pair r is kept only
+ * while z <= w_r, w_r = min(k * lambda_r, N), lambda_r = 2*pi / theta_r (Eq. 2, Eq. 3).
+ * Softmax, the P*V product and the online-softmax recurrence are the usual ones (Sec. 3.3).
+ *
+ * Conventions shared by every entry point
+ *   - All tensors are contiguous, row-major, with the shapes given below; bf16 unless stated.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *   - The caller owns every buffer.  The library allocates no device memory; scratch comes
+ *     from the workspace the caller binds with atf_bind_workspace().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
+ *     asynchronous with respect to the host unless stated.
+ *   - Every function returns an atf_status; nothing throws or aborts.  Arguments are checked
+ *     on the host before any launch.  atf_last_error() gives a text for the last failure of
+ *     the calling thread.
+ *   - Head dimension d is 64 or 128; Hq must be a multiple of Hkv; query head hq reads KV head
+ *     hq / (Hq/Hkv).  The softmax scale is 1/sqrt(d) (Eq. 1).  Pair r is dims (r, r + d/2)
+ *     ("half-split" RoPE layout).
+ */
+#ifndef ATFLASH_H
+#define ATFLASH_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int atf_status;
+enum {
+  ATF_OK = 0,
+  ATF_ERR_INVALID_ARG = 1, /* null pointer, bad shape, malformed table                      */
+  ATF_ERR_UNSUPPORTED = 2, /* valid request the library does not implement                   */
+  ATF_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (text in atf_last_error)      */
+  ATF_ERR_WORKSPACE = 4,   /* no workspace bound, or it is too small for this call            */
+  ATF_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out during an earlier launch     */
+};
+
+/* Modes (second argument of the *_ex calls).
+ * ATF_MODE_EXACT : the per-term definition (the predicate under Eq. 3 applied to every term).
+ * ATF_MODE_COARSE: the granularity the paper's ports run at (Sec. 3.3, Sec. 5, App. E).
+ *   Prefill: the live pair set is chosen per (128-query, 128-key) tile from the tile's nearest
+ *   cell and rounded outward to whole groups of 8 pairs counted from the low-frequency end;
+ *   the tile on the diagonal uses every pair.  Decode: per key, the first live pair is rounded
+ *   down to a multiple of 8 pairs (one 16-byte load per half row).                           */
+enum { ATF_MODE_EXACT = 0, ATF_MODE_COARSE = 1 };
+
+/* RoPE frequency scaling (Sec. 3.2: the table is built from the effective frequencies).
+ * kind 0: none.  kind 1: llama3-style - with lambda = 2*pi/theta and c = original_ctx, a pair
+ * with lambda < c/high_freq_factor keeps theta, one with lambda > c/low_freq_factor gets
+ * theta/factor, and in between theta' = (1-t)*theta/factor + t*theta with
+ * t = (c/lambda - low_freq_factor) / (high_freq_factor - low_freq_factor).                   */
+typedef struct {
+  int kind;
+  double factor, low_freq_factor, high_freq_factor;
+  int64_t original_ctx;
+} atf_scaling;
+
+/* Optional arguments of the *_ex calls.  Zero-initialise, then set what is needed. */
+typedef struct {
+  int mode;              /* ATF_MODE_EXACT or ATF_MODE_COARSE                                  */
+  uint64_t* kept_terms;  /* dev, [B*Hq] or NULL.  If set, the kernel ADDS to entry b*Hq+hq the
+                            number of (cell, pair) inner-product terms it executed for that head
+                            (Sec. 4 cost measure); the caller zeroes it beforehand.             */
+  float* lse;            /* decode only: dev, [B*Hq] fp32 natural-log LSE, or NULL              */
+  void* workspace;       /* dev scratch for this call, or NULL to use the bound workspace       */
+  size_t workspace_bytes;
+} atf_opts;
+
+/* Window table (Eq. 2, Eq. 3; effective frequencies per Sec. 3.2).  Host only, no GPU needed.
+ *   theta_r = base^(-2r/d) in IEEE double, scaled per `s` (NULL = none);
+ *   w_out[r] = floor(min(k * 2*pi/theta'_r, N)) for r in [0, d/2): the predicate "z <= w_r" on
+ *   integer distances only sees the integer part.  k = INFINITY gives w_out[r] = N.
+ *   theta_out (host, d/2 doubles) receives theta'_r if not NULL (the input atf_rope wants).
+ * Errors: ATF_ERR_INVALID_ARG for d odd or <= 0, N < 1, k < 0 or NaN, null w_out.             */
+atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_scaling* s,
+                            int64_t* w_out, double* theta_out);
+
+/* Half-split rotary embedding, in place (Sec. 3.1).
+ *   X: dev bf16 [B, H, N, d]; row n is rotated by the angle (pos0 + n) * theta[r] in pair r:
+ *   x'_r = x_r cos - x_{r+d/2} sin,  x'_{r+d/2} = x_{r+d/2} cos + x_r sin.
+ *   theta: host, d/2 doubles.  Angles and the rotation are evaluated in fp64 and rounded once
+ *   to bf16, so positions up to 2^20 and beyond keep full accuracy.                           */
+atf_status atf_rope(void* X, int B, int H, int64_t N, int d, const double* theta, int64_t pos0,
+                    void* stream);
+
+/* Prefill: windowed causal attention for all N query rows (Sec. 3.3, Fig. 3).
+ *   Q, O: dev bf16 [B, Hq, N, d];  K, V: dev bf16 [B, Hkv, N, d];  Q and K already rotated.
+ *   LSE: dev fp32 [B, Hq, N], natural log of the sum of exp(scaled score); may be NULL.
+ *   table: host int64 [d/2] from atf_window_table, non-decreasing in r and >= 0;
+ *          NULL = full attention (identical, bit for bit, to a table whose entries are all N).
+ *   A key with no live pair at all (z greater than every w_r) is dropped from the softmax.
+ *   causal must be 1: the paper defines the distance only for causal attention; 0 returns
+ *   ATF_ERR_UNSUPPORTED.  Needs a workspace of atf_workspace_bytes(ATF_OP_PREFILL, ...).
+ *   atf_prefill == atf_prefill_ex with opts = NULL (exact mode, no counters).                 */
+atf_status atf_prefill(const void* Q, const void* K, const void* V, void* O, float* LSE, int B,
+                       int Hq, int Hkv, int64_t N, int d, const int64_t* table, int causal,
+                       void* stream);
+atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B,
+                          int Hq, int Hkv, int64_t N, int d, const int64_t* table, int causal,
+                          const atf_opts* opts, void* stream);
+
+/* Decode: one new query token per sequence against a contiguous KV cache (Sec. 5; the last
+ * row of Fig. 3).  The cache already contains the new token; the query sits at position L-1,
+ * so key m is at distance z = L-1-m.
+ *   q, O: dev bf16 [B, Hq, d];  Kcache, Vcache: dev bf16 [B, Hkv, L, d] (the layout of K and V
+ *   in atf_prefill, so a prefill cache is read with no conversion).
+ *   Only the live low-frequency segments of each key row are read; V rows are read in full.
+ *   Needs a workspace of atf_workspace_bytes(ATF_OP_DECODE, ...).                             */
+atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, void* O, int B,
+                      int Hq, int Hkv, int64_t L, int d, const int64_t* table, void* stream);
+atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, void* O, int B,
+                         int Hq, int Hkv, int64_t L, int d, const int64_t* table,
+                         const atf_opts* opts, void* stream);
+
+/* Workspace.  The library keeps no allocation of its own: the caller allocates
+ * atf_workspace_bytes() bytes of device memory (256-byte aligned), zero-fills it once, and
+ * binds it (per process; the pointer is only stored).  One call at a time may use a given
+ * workspace; calls that overlap on the GPU need separate workspaces (atf_opts.workspace).     */
+enum { ATF_OP_PREFILL = 0, ATF_OP_DECODE = 1 };
+size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d);
+atf_status atf_bind_workspace(void* dev_ptr, size_t bytes);
+
+/* Reads (and clears) the device status word of the bound workspace; synchronises `stream`.
+ * Returns ATF_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last check.        */
+atf_status atf_check_status(void* stream);
+
+/* Text of the calling thread's last error ("" if none). Never NULL. */
+const char* atf_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATFLASH_H */

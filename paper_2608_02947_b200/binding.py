@@ -1,0 +1,213 @@
+"""ctypes binding of libatflash.so.  Argument marshalling only; every step runs in the library."""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+ATF_MODE_EXACT, ATF_MODE_COARSE = 0, 1
+ATF_OP_PREFILL, ATF_OP_DECODE = 0, 1
+
+
+class AtfError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"atflash error {code}: {text}")
+        self.code = code
+
+
+class _Scaling(C.Structure):
+    _fields_ = [("kind", C.c_int), ("factor", C.c_double), ("low_freq_factor", C.c_double),
+                ("high_freq_factor", C.c_double), ("original_ctx", C.c_int64)]
+
+
+class _Opts(C.Structure):
+    _fields_ = [("mode", C.c_int), ("kept_terms", C.c_void_p), ("lse", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+def lib_path():
+    return os.path.join(_HERE, "libatflash.so")
+
+
+_lib = None
+
+
+def lib():
+    """Loads libatflash.so (built by `python -m paper_2608_02947_b200.build`). Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    p = lib_path()
+    if not os.path.exists(p):
+        raise AtfError(-1, f"{p} is missing: build it with `python -m paper_2608_02947_b200.build` "
+                           "(there is no fallback implementation)")
+    L = C.CDLL(p)
+    vp, i, i64, dbl = C.c_void_p, C.c_int, C.c_int64, C.c_double
+    L.atf_window_table.argtypes = [dbl, i, dbl, i64, C.POINTER(_Scaling), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
+    L.atf_rope.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
+    L.atf_prefill.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, vp]
+    L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
+    L.atf_decode.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
+    L.atf_decode_ex.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), C.POINTER(_Opts), vp]
+    L.atf_workspace_bytes.argtypes = [i, i, i, i, i64, i]
+    L.atf_workspace_bytes.restype = C.c_size_t
+    L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
+    L.atf_check_status.argtypes = [vp]
+    L.atf_last_error.restype = C.c_char_p
+    for name in ("atf_window_table", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_decode", "atf_decode_ex",
+                 "atf_bind_workspace", "atf_check_status"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(code):
+    if code != 0:
+        raise AtfError(code, lib().atf_last_error().decode())
+
+
+def llama3_scaling(factor=32.0, low_freq_factor=1.0, high_freq_factor=4.0, original_ctx=8192):
+    return {"kind": "llama3", "factor": factor, "low_freq_factor": low_freq_factor,
+            "high_freq_factor": high_freq_factor, "original_ctx": original_ctx}
+
+
+def atf_window_table(base, d, k, N, scaling=None):
+    """Returns (W int64[d/2] tensor on the host, theta float64[d/2] tensor on the host)."""
+    h = max(d // 2, 1)
+    w = (C.c_int64 * h)()
+    th = (C.c_double * h)()
+    sc = None
+    if scaling is not None and scaling.get("kind", "none") != "none":
+        kind = {"llama3": 1}.get(scaling["kind"], 99)
+        sc = C.byref(_Scaling(kind, float(scaling["factor"]), float(scaling["low_freq_factor"]),
+                              float(scaling["high_freq_factor"]), int(scaling["original_ctx"])))
+    _check(lib().atf_window_table(float(base), int(d), float(k), int(N), sc, w, th))
+    return torch.tensor(list(w), dtype=torch.int64), torch.tensor(list(th), dtype=torch.float64)
+
+
+def _stream(t):
+    return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def _dev_bf16(t, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+        raise AtfError(1, f"{name} must be a contiguous CUDA bf16 tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+def _table_ptr(table, d):
+    if table is None:
+        return None, None
+    t = torch.as_tensor(table, dtype=torch.int64).cpu().contiguous()
+    if t.numel() != d // 2:
+        raise AtfError(1, f"table must have d/2 = {d // 2} entries")
+    arr = (C.c_int64 * t.numel())(*t.tolist())
+    return arr, arr
+
+
+_ws = None
+
+
+def atf_workspace_bytes(op, B, Hq, Hkv, N, d):
+    return int(lib().atf_workspace_bytes(op, B, Hq, Hkv, N, d))
+
+
+def ensure_workspace(nbytes, device):
+    """Keeps one zero-initialised device buffer bound as the library's workspace (grown on demand)."""
+    global _ws
+    if _ws is None or _ws.numel() < nbytes or _ws.device != torch.device(device):
+        _ws = None
+        _ws = torch.zeros(max(nbytes, 256), dtype=torch.uint8, device=device)
+        _check(lib().atf_bind_workspace(C.c_void_p(_ws.data_ptr()), _ws.numel()))
+    return _ws
+
+
+def atf_rope(X, theta, pos0=0):
+    """In-place half-split RoPE of X [B,H,N,d] (CUDA bf16) at positions pos0..pos0+N-1."""
+    _dev_bf16(X, "X")
+    B, H, N, d = X.shape
+    th = torch.as_tensor(theta, dtype=torch.float64).cpu()
+    arr = (C.c_double * th.numel())(*th.tolist())
+    _check(lib().atf_rope(C.c_void_p(X.data_ptr()), B, H, N, d, arr, int(pos0), _stream(X)))
+    return X
+
+
+def _opts(mode, kept_terms, lse):
+    if mode == ATF_MODE_EXACT and kept_terms is None and lse is None:
+        return None
+    o = _Opts()
+    o.mode = int(mode)
+    o.kept_terms = kept_terms.data_ptr() if kept_terms is not None else None
+    o.lse = lse.data_ptr() if lse is not None else None
+    o.workspace = None
+    o.workspace_bytes = 0
+    return o
+
+
+def _host_roundtrip(tensors):
+    """For host inputs: pinned staging + device copies (the end-to-end path of the binding)."""
+    return [t.pin_memory().to("cuda", non_blocking=True) if not t.is_cuda else t for t in tensors]
+
+
+def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
+                O=None, LSE=None):
+    """Windowed causal attention.  Q [B,Hq,N,d], K/V [B,Hkv,N,d] bf16, already rotated.
+
+    Device tensors are used in place; host tensors are copied to the current CUDA device and
+    the results copied back (host in -> host out).  Returns (O, LSE) (LSE None if not asked).
+    """
+    on_host = not Q.is_cuda
+    if on_host:
+        Q, K, V = _host_roundtrip([Q, K, V])
+    for t, nm in ((Q, "Q"), (K, "K"), (V, "V")):
+        _dev_bf16(t, nm)
+    B, Hq, N, d = Q.shape
+    Hkv = K.shape[1]
+    if K.shape != (B, Hkv, N, d) or V.shape != K.shape:
+        raise AtfError(1, "K and V must be [B,Hkv,N,d] matching Q")
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None and return_lse:
+        LSE = torch.empty((B, Hq, N), dtype=torch.float32, device=Q.device)
+    ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL, B, Hq, Hkv, N, d), Q.device)
+    tab, _keep = _table_ptr(table, d)
+    o = _opts(mode, kept_terms, None)
+    lse_ptr = C.c_void_p(LSE.data_ptr()) if LSE is not None else None
+    _check(lib().atf_prefill_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+                                C.byref(o) if o is not None else None, _stream(Q)))
+    if on_host:
+        return O.cpu(), (LSE.cpu() if LSE is not None else None)
+    return O, LSE
+
+
+def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=False, O=None):
+    """One decode step: q [B,Hq,d] at position L-1 against Kcache/Vcache [B,Hkv,L,d] (bf16)."""
+    on_host = not q.is_cuda
+    if on_host:
+        q, Kcache, Vcache = _host_roundtrip([q, Kcache, Vcache])
+    for t, nm in ((q, "q"), (Kcache, "Kcache"), (Vcache, "Vcache")):
+        _dev_bf16(t, nm)
+    B, Hq, d = q.shape
+    Hkv, L = Kcache.shape[1], Kcache.shape[2]
+    if Kcache.shape != (B, Hkv, L, d) or Vcache.shape != Kcache.shape:
+        raise AtfError(1, "Kcache and Vcache must be [B,Hkv,L,d] matching q")
+    if O is None:
+        O = torch.empty_like(q)
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
+    ensure_workspace(atf_workspace_bytes(ATF_OP_DECODE, B, Hq, Hkv, L, d), q.device)
+    tab, _keep = _table_ptr(table, d)
+    o = _opts(mode, kept_terms, lse)
+    _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
+                               C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,
+                               C.byref(o) if o is not None else None, _stream(q)))
+    if on_host:
+        return (O.cpu(), lse.cpu()) if return_lse else O.cpu()
+    return (O, lse) if return_lse else O
+
+
+def check_status():
+    _check(lib().atf_check_status(C.c_void_p(torch.cuda.current_stream().cuda_stream)))

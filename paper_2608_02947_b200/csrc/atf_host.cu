@@ -1,0 +1,116 @@
+// Host-side parts of the atflash library: window table (Eq. 2, Eq. 3, Sec. 3.2), error
+// text, workspace binding and the device status word.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "atf_common.cuh"
+
+static thread_local char g_err[512] = "";
+static AtfWorkspace g_ws = {nullptr, 0};
+
+atf_status atf_fail(atf_status code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+AtfWorkspace atf_bound_workspace() { return g_ws; }
+
+int atf_decode_num_splits(int B, int Hkv, int64_t L) {
+  int64_t groups = (int64_t)B * Hkv;
+  int64_t want = (ATF_DECODE_TARGET_CTAS + groups - 1) / groups;
+  int64_t most = (L + ATF_DECODE_MIN_SPLIT - 1) / ATF_DECODE_MIN_SPLIT;
+  if (want > most) want = most;
+  if (want < 1) want = 1;
+  return (int)want;
+}
+
+// Checks a caller's table (host, d/2 entries; NULL = full attention) and converts it to the
+// int32 form the kernels take.  The live pair set at a distance must be a contiguous
+// low-frequency slice (Sec. 3.3), which needs widths that do not decrease with r.
+atf_status atf_validate_table(const char* who, const int64_t* table, int d, int64_t N, AtfTable* out) {
+  const int h = d / 2;
+  for (int r = 0; r < ATF_MAX_PAIRS; ++r) out->w[r] = 0x7FFFFFFF;
+  for (int r = 0; r < h; ++r) {
+    int64_t w = table ? table[r] : N;
+    if (w < 0) return atf_fail(ATF_ERR_INVALID_ARG, "%s: table[%d] is negative", who, r);
+    if (table && r > 0 && table[r] < table[r - 1])
+      return atf_fail(ATF_ERR_UNSUPPORTED, "%s: table must be non-decreasing in r (entry %d)", who, r);
+    if (w > N) w = N;  // distances never exceed N-1, so clipping changes nothing
+    out->w[r] = (int32_t)w;
+  }
+  return ATF_OK;
+}
+
+size_t atf_decode_workspace_bytes(int B, int Hq, int Hkv, int64_t L, int d);
+size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d);
+
+extern "C" {
+
+size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d) {
+  if (B < 1 || Hq < 1 || Hkv < 1 || N < 1 || (d != 64 && d != 128)) return 0;
+  if (op == ATF_OP_PREFILL) return atf_prefill_workspace_bytes(B, Hq, Hkv, N, d);
+  if (op == ATF_OP_DECODE) return atf_decode_workspace_bytes(B, Hq, Hkv, N, d);
+  return 0;
+}
+
+const char* atf_last_error(void) { return g_err; }
+
+atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_scaling* s,
+                            int64_t* w_out, double* theta_out) {
+  if (d <= 0 || (d & 1)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: d must be even and positive (got %d)", d);
+  if (N < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: N must be >= 1");
+  if (!(k >= 0.0)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: k must be >= 0 (INFINITY = full attention)");
+  if (!(base > 1.0)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: base must be > 1");
+  if (!w_out) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: w_out is NULL");
+  if (s && s->kind != 0 && s->kind != 1) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_window_table: unknown scaling kind %d", s->kind);
+  const double two_pi = 2.0 * M_PI;
+  const int h = d / 2;
+  for (int r = 0; r < h; ++r) {
+    double theta = std::pow(base, -2.0 * (double)r / (double)d);
+    if (s && s->kind == 1) {
+      const double lam = two_pi / theta;
+      const double c = (double)s->original_ctx;
+      if (lam < c / s->high_freq_factor) {
+        // short wavelength: unchanged
+      } else if (lam > c / s->low_freq_factor) {
+        theta = theta / s->factor;
+      } else {
+        const double t = (c / lam - s->low_freq_factor) / (s->high_freq_factor - s->low_freq_factor);
+        theta = (1.0 - t) * theta / s->factor + t * theta;
+      }
+    }
+    if (theta_out) theta_out[r] = theta;
+    const double w = k * (two_pi / theta);
+    w_out[r] = (w < (double)N) ? (int64_t)std::floor(w) : N;
+  }
+  return ATF_OK;
+}
+
+atf_status atf_bind_workspace(void* dev_ptr, size_t bytes) {
+  if (dev_ptr && ((uintptr_t)dev_ptr & 255)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_bind_workspace: pointer must be 256-byte aligned");
+  if (dev_ptr && bytes < ATF_WS_HEADER) return atf_fail(ATF_ERR_WORKSPACE, "atf_bind_workspace: workspace smaller than its header");
+  g_ws.ptr = dev_ptr;
+  g_ws.bytes = dev_ptr ? bytes : 0;
+  return ATF_OK;
+}
+
+atf_status atf_check_status(void* stream) {
+  if (!g_ws.ptr) return atf_fail(ATF_ERR_WORKSPACE, "atf_check_status: no workspace bound");
+  unsigned int st[2] = {0, 0};
+  cudaStream_t s = (cudaStream_t)stream;
+  ATF_CUDA_CHECK(cudaMemcpyAsync(st, g_ws.ptr, sizeof(st), cudaMemcpyDeviceToHost, s));
+  ATF_CUDA_CHECK(cudaStreamSynchronize(s));
+  if (st[0] != 0) {
+    ATF_CUDA_CHECK(cudaMemsetAsync(g_ws.ptr, 0, sizeof(st), s));
+    ATF_CUDA_CHECK(cudaStreamSynchronize(s));
+    return atf_fail(ATF_ERR_TIMEOUT, "a kernel gave up a bounded wait (code %u at site %u)", st[0], st[1]);
+  }
+  return ATF_OK;
+}
+
+}  // extern "C"
