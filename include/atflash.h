@@ -120,7 +120,9 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
 
 /* Workspace.  The library keeps no allocation of its own: the caller allocates
  * atf_workspace_bytes() bytes of device memory (256-byte aligned), zero-fills it once, and
- * binds it (per process; the pointer is only stored).  One call at a time may use a given
+ * binds it (per process; the pointer is only stored).  A workspace sized for the largest call
+ * serves prefill and decode in turn: its first 64.25 KiB (status words and decode's split
+ * counters, which the kernels leave zeroed) are never used as scratch.  One call at a time may use a given
  * workspace; calls that overlap on the GPU need separate workspaces (atf_opts.workspace).     */
 enum { ATF_OP_PREFILL = 0, ATF_OP_DECODE = 1 };
 size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d);

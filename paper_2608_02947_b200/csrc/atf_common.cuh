@@ -25,13 +25,14 @@ struct AtfTable {
   int32_t w[ATF_MAX_PAIRS];
 };
 
-// Workspace header (first 256 bytes of every workspace).
-struct AtfWsHeader {
-  unsigned int status;  // 0 = fine; otherwise a code written by a kernel that gave up a wait
-  unsigned int where;   // which wait
-  unsigned int pad[62];
-};
-constexpr size_t ATF_WS_HEADER = 256;
+// Workspace header, common to every operation so that one workspace can serve prefill and
+// decode in turn: 256 bytes of status words (word 0: non-zero once a kernel gave up a bounded
+// wait; word 1: which wait), then the split counters of decode (one per (batch, KV head);
+// they must be zero between launches, which the decode kernel restores itself).  Nothing else
+// ever writes into the header.
+constexpr size_t ATF_WS_STATUS_BYTES = 256;
+constexpr int ATF_WS_COUNTER_SLOTS = 16384;
+constexpr size_t ATF_WS_HEADER = ATF_WS_STATUS_BYTES + (size_t)ATF_WS_COUNTER_SLOTS * 4;
 
 struct AtfWorkspace {
   void* ptr;

@@ -352,8 +352,7 @@ static size_t decode_ws_bytes(int B, int Hq, int Hkv, int64_t L, int d) {
   const int ns = atf_decode_num_splits(B, Hkv, L);
   size_t partials = (size_t)B * Hq * ns * (d + 2) * sizeof(float);
   partials = (partials + 255) & ~(size_t)255;
-  size_t counters = ((size_t)B * Hkv * sizeof(unsigned int) + 255) & ~(size_t)255;
-  return ATF_WS_HEADER + counters + partials;
+  return ATF_WS_HEADER + partials;
 }
 size_t atf_decode_workspace_bytes(int B, int Hq, int Hkv, int64_t L, int d) { return decode_ws_bytes(B, Hq, Hkv, L, d); }
 
@@ -365,7 +364,8 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: bad shape");
   if (Hq % Hkv) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: Hq must be a multiple of Hkv");
   if (L * (int64_t)d >= (1ll << 31)) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: L*d must be below 2^31");
-  if (B > 65535 || Hkv > 65535) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: B and Hkv must be <= 65535");
+  if (B > 65535 || Hkv > 65535 || (int64_t)B * Hkv > ATF_WS_COUNTER_SLOTS)
+    return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: B*Hkv must be <= %d", ATF_WS_COUNTER_SLOTS);
   if (((uintptr_t)q | (uintptr_t)Kcache | (uintptr_t)Vcache | (uintptr_t)O) & 15)
     return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: pointers must be 16-byte aligned");
   const int mode = opts ? opts->mode : ATF_MODE_EXACT;
@@ -398,9 +398,8 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.keys_per_split = (int)kps;
   P.nsplit = (int)((L + kps - 1) / kps);  // drop splits the rounding emptied
   char* base = (char*)ws.ptr;
-  P.counters = (unsigned int*)(base + ATF_WS_HEADER);
-  const size_t counters = ((size_t)B * Hkv * sizeof(unsigned int) + 255) & ~(size_t)255;
-  P.partials = (float*)(base + ATF_WS_HEADER + counters);
+  P.counters = (unsigned int*)(base + ATF_WS_STATUS_BYTES);
+  P.partials = (float*)(base + ATF_WS_HEADER);
   cudaStream_t s = (cudaStream_t)stream;
   const bool count = P.kept != nullptr;
   return d == 64 ? dispatch_group<64>(Hq / Hkv, P, t, B, mode, count, s)

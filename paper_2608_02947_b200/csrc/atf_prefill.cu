@@ -240,15 +240,17 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       cnt += (unsigned long long)depth * (unsigned long long)ncols;
     }
 
-    // ---- scale, causal mask, drop keys no pair reaches, online softmax ----
-    const bool need_mask = (dt == 0) || (zmax > Wmax);
+    // ---- scale, causal mask, drop keys no pair reaches (exact mode: per cell; coarse mode
+    //      decides per tile, which the loop exit above already did), online softmax ----
+    const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
+    const bool need_mask = (dt == 0) || (zmax > zdrop);
     float mx = -INFINITY;
     if (need_mask) {
       const int zrow = n - m0;
 #pragma unroll
       for (int c = 0; c < T; ++c) {
         const int z = zrow - c;
-        s[c] = (z >= 0 && z <= Wmax) ? s[c] * kScaleLog2 : -INFINITY;
+        s[c] = (z >= 0 && z <= zdrop) ? s[c] * kScaleLog2 : -INFINITY;
         mx = fmaxf(mx, s[c]);
       }
     } else {
