@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the windowed-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+One step = one pass of the whole hot path over one batch of seeded synthetic input:
+window table (host) -> RoPE of Q and K -> windowed causal prefill -> one windowed decode step
+against the K/V just written.  The default workload is the Llama-3.2-3B attention-layer shape at
+128K tokens (the configuration the headline metric is quoted on).  Prints ONE JSON line.
+
+With --gpus N under torchrun every rank runs an independent replica (the path has no exchange
+step); rank 0 reports the aggregate with the max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import atf_inputs as gen  # noqa: E402
+
+METRIC = "prefill executed TFLOP/s at 128K (with ms, decode us/step and HBM GB/s alongside)"
+
+
+def workload_by_name(name):
+    if name == "llama3b-128k":
+        return gen.llama32_3b(131072, B=1, seed_off=6)
+    if name == "llama3b-32k":
+        return gen.llama32_3b(32768, B=1, seed_off=5)
+    if name == "llama3b-8k":
+        return gen.llama32_3b(8192, B=1, seed_off=4)
+    if name == "qwen05b-32k":
+        return gen.qwen05b(32768)
+    if name == "qwen7b-1m":
+        return gen.qwen7b_1m(1 << 20)
+    if name == "tiny":
+        return gen.tiny()
+    raise SystemExit(f"unknown workload {name}")
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops"],
+                "bf16_tflops_sustained": j.get("bf16_tflops_sustained", j["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---- work accounting (definitions only: Sec. 4's term count turned into FLOPs and bytes) ----
+def kept_terms_prefill(W, N):
+    tot = 0
+    for w in W:
+        w = int(w)
+        a = min(w, N - 1)
+        tot += (a + 1) * (a + 2) // 2 + max(0, N - 1 - w) * (w + 1)
+    return tot
+
+
+def kept_terms_decode(W, L):
+    return sum(min(int(w), L - 1) + 1 for w in W)
+
+
+def prefill_flops(wl, W):
+    cells = wl.N * (wl.N + 1) // 2
+    executed = wl.B * wl.Hq * (4 * kept_terms_prefill(W, wl.N) + 2 * wl.d * cells)
+    effective = wl.B * wl.Hq * 4 * wl.d * cells
+    return executed, effective
+
+
+def decode_bytes(wl, W, windowed=True):
+    L = wl.N
+    kept = kept_terms_decode(W, L) if windowed else (wl.d // 2) * L
+    return wl.B * wl.Hkv * (4 * kept + 2 * wl.d * L)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [v for v in sm if mx and v > 0]
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def run_ours(args):
+    import paper_2608_02947_b200 as atf
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    atf.lib()  # fails loudly if the CUDA library is missing
+
+    wl = workload_by_name(args.workload)
+    pk = peaks()
+    Q0, K0, V = gen.prefill_inputs(wl, device=dev)  # un-rotated, on the device
+    Qg, Kg = Q0.clone(), K0.clone()
+    O = torch.empty_like(Qg)
+    LSE = torch.empty((wl.B, wl.Hq, wl.N), dtype=torch.float32, device=dev)
+    qd = torch.empty((wl.B, wl.Hq, wl.d), dtype=torch.bfloat16, device=dev)
+    Od = torch.empty_like(qd)
+    nbytes = max(atf.atf_workspace_bytes(0, wl.B, wl.Hq, wl.Hkv, wl.N, wl.d),
+                 atf.atf_workspace_bytes(1, wl.B, wl.Hq, wl.Hkv, wl.N, wl.d))
+    atf.ensure_workspace(nbytes, dev)
+
+    t_rope, t_pre, t_dec, t_step = [], [], [], []
+
+    def step(timed):
+        e = [ev() for _ in range(5)]
+        e[0].record()
+        W, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+        Qg.copy_(Q0)
+        Kg.copy_(K0)
+        e[1].record()
+        atf.atf_rope(Qg, theta)
+        atf.atf_rope(Kg, theta)
+        e[2].record()
+        atf.atf_prefill(Qg, Kg, V, table=W, O=O, LSE=LSE)
+        e[3].record()
+        qd.copy_(Qg[:, :, -1])
+        atf.atf_decode(qd, Kg, V, table=W, O=Od)
+        e[4].record()
+        if timed:
+            torch.cuda.synchronize()
+            t_rope.append(e[1].elapsed_time(e[2]))
+            t_pre.append(e[2].elapsed_time(e[3]))
+            t_dec.append(e[3].elapsed_time(e[4]))
+        return W
+
+    for _ in range(args.warmup):
+        W = step(False)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    torch.cuda.synchronize()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for _ in range(args.steps):
+        W = step(True)
+    t1.record()
+    torch.cuda.synchronize()
+    total_ms = t0.elapsed_time(t1)
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    atf.binding.check_status()
+    if rank != 0:
+        return
+
+    if args.profile_only:
+        print(json.dumps({"profile_only": True, "workload": args.workload, "ms_per_step": total_ms / args.steps,
+                          "prefill_ms": statistics.median(t_pre), "decode_us": statistics.median(t_dec) * 1e3}))
+        return
+    Wl = W.tolist()
+    executed, effective = prefill_flops(wl, Wl)
+    pre_ms = statistics.median(t_pre)
+    dec_ms = statistics.median(t_dec)
+    rope_ms = statistics.median(t_rope)
+    step_ms = total_ms / args.steps
+    # the step's own work, without the two device copies that restore the un-rotated inputs
+    work_ms = rope_ms + pre_ms + dec_ms
+
+    # ---- the same library at k = infinity (full attention) ----
+    full_pre, full_dec = [], []
+    for _ in range(2):
+        a, b_, c = ev(), ev(), ev()
+        a.record()
+        atf.atf_prefill(Qg, Kg, V, table=None, O=O, LSE=LSE)
+        b_.record()
+        atf.atf_decode(qd, Kg, V, table=None, O=Od)
+        c.record()
+        torch.cuda.synchronize()
+        full_pre.append(a.elapsed_time(b_))
+        full_dec.append(b_.elapsed_time(c))
+    full_pre_ms, full_dec_ms = min(full_pre), statistics.median(full_dec)
+
+    # ---- decode alone, cycling a KV pool of >= 512 MiB so that no read hits L2 from an earlier one ----
+    kv_bytes = 2 * Kg.numel() * 2
+    npool = max(2, math.ceil((512 << 20) / kv_bytes) + 1)
+    pool = [(Kg, V)] + [(Kg.clone(), V.clone()) for _ in range(npool - 1)]
+    dec_t = {True: [], False: []}
+    for windowed in (True, False):
+        for i in range(8 + 40):
+            Kc, Vc = pool[i % npool]
+            a, b_ = ev(), ev()
+            a.record()
+            atf.atf_decode(qd, Kc, Vc, table=W if windowed else None, O=Od)
+            b_.record()
+            torch.cuda.synchronize()
+            if i >= 8:
+                dec_t[windowed].append(a.elapsed_time(b_) * 1e3)
+    dec_us, dec_full_us = statistics.median(dec_t[True]), statistics.median(dec_t[False])
+    del pool
+    dbytes = decode_bytes(wl, Wl, True)
+    dbytes_full = decode_bytes(wl, Wl, False)
+
+    # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region ----
+    hQ, hK, hV = (t.cpu().pin_memory() for t in (Qg, Kg, V))
+    e2e_t = []
+    for i in range(3):
+        torch.cuda.synchronize()
+        ta = time.perf_counter()
+        Oh, Lh = atf.atf_prefill(hQ, hK, hV, table=W)
+        torch.cuda.synchronize()
+        if i:
+            e2e_t.append((time.perf_counter() - ta) * 1e3)
+    e2e_ms = statistics.median(e2e_t)
+    h2d = (hQ.numel() + hK.numel() + hV.numel()) * 2
+    d2h = Oh.numel() * 2 + Lh.numel() * 4
+
+    # ---- CPU baseline: the oracle as it stands on a bounded sample of the same workload ----
+    cpu = cpu_baseline(wl, budget_s=args.cpu_budget)
+
+    total_exec = executed  # decode's FLOPs are ~1e-6 of the step
+    out = {
+        "metric": METRIC, "value": world * total_exec / (pre_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name} attention layer B={wl.B} Hq={wl.Hq} Hkv={wl.Hkv} d={wl.d} N=L={wl.N} k={wl.k} "
+                               f"({'llama3-scaled' if wl.scaling else 'raw'} RoPE base {wl.base:g}), exact mode",
+                   "step": "window_table + rope(Q,K) + prefill + decode", "l2": "inputs larger than L2; decode cycles a KV pool",
+                   "replicas": world},
+        "prefill_ms": pre_ms, "prefill_executed_tflops": executed / (pre_ms * 1e-3) / 1e12,
+        "prefill_effective_tflops": effective / (pre_ms * 1e-3) / 1e12,
+        "prefill_full_ms": full_pre_ms, "prefill_speedup_vs_full": full_pre_ms / pre_ms,
+        "prefill_full_tflops": effective / (full_pre_ms * 1e-3) / 1e12,
+        "prefill_ceiling": effective / executed,
+        "rope_ms": rope_ms, "work_ms": work_ms,
+        "decode_us": dec_us, "decode_gbs": dbytes / (dec_us * 1e-6) / 1e9,
+        "decode_full_us": dec_full_us, "decode_full_gbs": dbytes_full / (dec_full_us * 1e-6) / 1e9,
+        "decode_speedup_vs_full": dec_full_us / dec_us, "decode_in_step_us": dec_ms * 1e3,
+        "frac_of_nominal": {"prefill_executed_of_2250": executed / (pre_ms * 1e-3) / 1e12 / 2250.0,
+                            "decode_of_8000": dbytes / (dec_us * 1e-6) / 1e9 / 8000.0},
+        "roofline": {"bound": "tensor", "achieved": executed / (pre_ms * 1e-3) / 1e12,
+                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": executed / (pre_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], "traffic": None,
+                     "kernel": "atf_prefill_kernel (+2 repack launches, <1% of the time)",
+                     "peak_source": f"{pk['source']} sustained bf16 GEMM"},
+        "roofline_decode": {"bound": "hbm", "achieved": dbytes / (dec_us * 1e-6) / 1e9, "peak": pk["hbm_gbs"],
+                            "unit": "GB/s", "frac": dbytes / (dec_us * 1e-6) / 1e9 / pk["hbm_gbs"], "traffic": None,
+                            "kernel": "atf_decode_kernel", "peak_source": f"{pk['source']} copy bandwidth"},
+        "e2e": {"value": executed / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "what": "atf_prefill on pinned host tensors: H2D of Q,K,V + kernels + D2H of O,LSE"},
+        "gpu_launches": 6 * args.steps,
+        "clocks": clocks,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+
+
+def cpu_baseline(wl, budget_s=15.0):
+    """Times oracle/ (fp64 NumPy, as it stands) on sampled query rows of the same workload."""
+    import numpy as np
+
+    from oracle import atf_oracle as orc
+    W, theta = orc.window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+    rng = np.random.default_rng(wl.seed)
+    # one head's worth of rotated-looking data (the cost does not depend on values)
+    K = orc.round_to_bf16(rng.standard_normal((wl.N, wl.d)))
+    V = orc.round_to_bf16(rng.standard_normal((wl.N, wl.d)))
+    Q = orc.round_to_bf16(rng.standard_normal((wl.N, wl.d)))
+    rows, flops, t0 = 0, 0, time.perf_counter()
+    while time.perf_counter() - t0 < budget_s:
+        n = int(rng.integers(0, wl.N))
+        orc.attention_rows(Q, K, V, W, [n])
+        rows += 1
+        flops += 4 * orc.kept_terms_row(W, n) + 2 * wl.d * (n + 1)
+    dt = time.perf_counter() - t0
+    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+            "sample": f"{rows} random query rows of one head of the {wl.N}-token workload in {dt:.1f} s "
+                      f"(fp64 NumPy, single thread); executed FLOPs of those rows / time",
+            "host_cores_available": os.cpu_count()}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload_by_name(args.workload)
+    vals = []
+    per = max(3.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        c = cpu_baseline(wl, budget_s=per)
+        if i >= args.warmup:
+            vals.append(c)
+    v = statistics.median([c["value"] for c in vals])
+    out = {"impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{wl.name} attention layer N={wl.N} (bounded sample of query rows per step)"},
+           "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": 1, "kind": "oracle", "sample": vals[-1]["sample"]},
+           "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--workload", default="llama3b-128k")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--profile-only", action="store_true",
+                    help="run only the warm-up and timed steps (for ncu captures); prints a short line")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
