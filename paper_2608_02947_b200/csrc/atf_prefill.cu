@@ -272,19 +272,14 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
     l_run = l_run * alpha + psum;
 
-    // ---- P (bf16) to shared memory, K-major, 128-byte swizzle ----
+    // ---- P (bf16) into tensor memory, over the first 64 columns of S: column c of a lane
+    //      holds keys 2c (low half) and 2c+1 (high half) of that query row ----
+    {
+      uint32_t pk[64];
 #pragma unroll
-    for (int kb = 0; kb < 2; ++kb) {
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const float* sp = s + kb * 64 + ch * 8;
-        uint4 v;
-        v.x = pack_bf16x2(sp[0], sp[1]);
-        v.y = pack_bf16x2(sp[2], sp[3]);
-        v.z = pack_bf16x2(sp[4], sp[5]);
-        v.w = pack_bf16x2(sp[6], sp[7]);
-        *reinterpret_cast<uint4*>(smem_gen + SM::P_OFF + kb * BLK_BYTES + sw128_offset(row, ch)) = v;
-      }
+      for (int c = 0; c < 64; ++c) pk[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
+      tc_st32(tS + lane_off, pk);
+      tc_st32(tS + lane_off + 32, pk + 32);
     }
     // ---- rescale O ----
     if (!first) {
@@ -297,9 +292,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
         tc_st32(tO + lane_off + q4 * 32, o);
       }
-      tc_wait_st();
     }
-    fence_proxy_async_smem();
+    tc_wait_st();
     tc_fence_before();
     __syncthreads();
 
@@ -308,9 +302,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < T / 16; ++ks) {
-        const uint64_t da = make_smem_desc_sw128(sP + (ks >> 2) * BLK_BYTES + (ks & 3) * 32, 16, 1024);
         const uint64_t db = make_smem_desc_sw128(sV + ks * 2048, BLK_BYTES, 1024);
-        tc_mma_ss(tO, da, db, IDESC_PV, (first && ks == 0) ? 0u : 1u);
+        tc_mma_ts(tO, tS + ks * 8, db, IDESC_PV, (first && ks == 0) ? 0u : 1u);
       }
       tc_commit(bar_mma);
     }
