@@ -8,12 +8,16 @@
 // PREFIX of the columns, so "advance the start of the pair loop" becomes "contract over the
 // first few 16-column MMA steps", and the K columns beyond the prefix are not loaded.
 //
-// Kernel.  One CTA owns a 128-row query tile of one head and walks the key tiles from the
-// diagonal outwards.  Per key tile: TMA brings K (the live 64-column blocks) and V into
-// 128-byte-swizzled shared memory; tcgen05.mma accumulates S = Q K^T over the live depth into
-// tensor memory; the four warps read S (one row per thread), finish the window rule, apply
-// the causal mask and the online softmax, rescale O in tensor memory, write P as bf16 to
-// shared memory; tcgen05.mma accumulates O += P V.
+// Kernel.  One CTA owns 256 query rows of one head as two 128-row tiles, A (rows 256i..) and
+// B (the next 128), and walks the key tiles from B's diagonal outwards.  Warp roles:
+//   warp 0      TMA producer: Q once, then K (live 64-column blocks only) and V tiles into
+//               two-stage rings of 128-byte-swizzled shared memory;
+//   warp 1      MMA issuer (one thread): S_X = Q_X K^T over the live depth into tensor memory,
+//               O_X += P_X V with P read from tensor memory; the two query tiles alternate
+//               so that the tensor pipe works on one while the other is in its softmax;
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one query row per thread:
+//               read S, finish the window rule, mask, online softmax with lazy rescaling of
+//               O, write P (bf16) over S in tensor memory.
 //
 // Exact mode (the per-term definition).  For a tile at tile distance D the cells span
 // distances [z_min, z_max].  Pairs with w >= z_max are live in every cell: they are the MMA
@@ -28,8 +32,11 @@
 
 namespace {
 
-constexpr int T = 128;           // query rows and key columns per tile
+constexpr int T = 128;              // query rows per tile and key columns per tile
 constexpr int BLK_BYTES = T * 128;  // one [128 x 64] bf16 block, 128-byte rows
+constexpr int KS = 2, VS = 2;       // ring depths
+constexpr int PF_THREADS = 384;
+constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag behind
 
 struct PrefillParams {
   const __nv_bfloat16* Qp;  // pair-interleaved copy of Q, [B*Hq, N, D]
@@ -43,14 +50,17 @@ struct PrefillParams {
 template <int D>
 struct PrefillSmem {
   static constexpr int NB = D / 64;  // 64-column blocks per tile row
-  static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = Q_OFF + NB * BLK_BYTES;
-  static constexpr int V_OFF = K_OFF + NB * BLK_BYTES;
-  static constexpr int P_OFF = V_OFF + NB * BLK_BYTES;
-  static constexpr int BAR_OFF = P_OFF + 2 * BLK_BYTES;
-  static constexpr int TOTAL = BAR_OFF + 64;
+  static constexpr int TILE = NB * BLK_BYTES;
+  static constexpr int Q_OFF = 0;  // tile A, then tile B
+  static constexpr int K_OFF = Q_OFF + 2 * TILE;
+  static constexpr int V_OFF = K_OFF + KS * TILE;
+  static constexpr int BAR_OFF = V_OFF + VS * TILE;
+  static constexpr int TOTAL = BAR_OFF + 256;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment
 };
+// barrier slots (8 bytes each) inside the BAR area
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13,
+       B_QZ = 15, B_COUNT = 17 };
 
 __global__ void __launch_bounds__(256)
 atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D) {
@@ -72,22 +82,49 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
   *reinterpret_cast<uint4*>(Y + row * D + 8 * t) = *reinterpret_cast<const uint4*>(out);
 }
 
-__device__ __forceinline__ int count_ge(const int* w, int H, int z) {
-  // number of pairs whose window reaches distance z (w is non-decreasing)
-  int n = 0;
-  for (int r = 0; r < H; ++r) n += (w[r] >= z) ? 1 : 0;
-  return n;
+// Live-pair bookkeeping for a tile at tile distance dt (tiles of 128, aligned at 0): cells
+// span distances [zmin, zmax].  w[] is non-decreasing, so the pairs reaching a distance z are
+// r >= r0(z), and r0 only grows with dt: the cursors are advanced, never rewound.
+struct TileSched {
+  int r_any = 0, r_all = 0;  // first pair live in some cell / in every cell
+  __device__ __forceinline__ void advance(const int* w, int H, int dt) {
+    const int zmin = dt == 0 ? 0 : (dt - 1) * T + 1;
+    const int zmax = (dt + 1) * T - 1;
+    while (r_any < H && w[r_any] < zmin) ++r_any;
+    while (r_all < H && w[r_all] < zmax) ++r_all;
+  }
+};
+template <int MODE>
+__device__ __forceinline__ int tile_depth(int H, int p_any, int p_all, int dt) {
+  if (MODE == ATF_MODE_EXACT) return p_all;
+  return dt == 0 ? H : min(H, (p_any + 7) / 8 * 8);
+}
+
+// Bounded wait that also gives up as soon as another role of the CTA has given up.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > ATF_WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
 }
 
 template <int D, int MODE, bool COUNT>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(PF_THREADS, 1)
 atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ PrefillParams P,
                    const __grid_constant__ AtfTable table) {
   using SM = PrefillSmem<D>;
   constexpr int H = D / 2;
   constexpr int NB = D / 64;
-  constexpr uint32_t TMEM_COLS = 256;
+  constexpr uint32_t TMEM_COLS = 512;
   constexpr uint32_t IDESC_QK = make_idesc_bf16(128, T, 0, 0);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(128, D, 0, 1);
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
@@ -95,26 +132,39 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sQ = smem_base + SM::Q_OFF, sK = smem_base + SM::K_OFF, sV = smem_base + SM::V_OFF,
-                 sP = smem_base + SM::P_OFF;
-  const uint32_t bar_q = smem_base + SM::BAR_OFF, bar_kv = bar_q + 8, bar_mma = bar_q + 16;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + SM::BAR_OFF + 32);
+  const uint32_t sQ = smem_base + SM::Q_OFF, sK = smem_base + SM::K_OFF, sV = smem_base + SM::V_OFF;
+  const uint32_t bars = smem_base + SM::BAR_OFF;
+  auto bar = [&](int slot) { return bars + 8u * (uint32_t)slot; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + SM::BAR_OFF + 8 * B_COUNT);
   __shared__ int sW[ATF_MAX_PAIRS];
+  __shared__ int s_abort;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int nqt = (P.N + T - 1) / T;
-  const int it = nqt - 1 - (int)blockIdx.x;  // longest rows first
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int npt = (P.N + 2 * T - 1) / (2 * T);
+  const int ip = npt - 1 - (int)blockIdx.x;  // longest rows first
   const int hq = blockIdx.y, b = blockIdx.z;
   const int bhq = b * P.Hq + hq;
   const int bhk = b * P.Hkv + hq / (P.Hq / P.Hkv);
-  const int row = tid;
-  const int n = it * T + row;
+  const int itA = 2 * ip, itB = 2 * ip + 1;
 
   if (tid < H) sW[tid] = table.w[tid];
   if (tid == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_kv, 1);
-    mbar_init(bar_mma, 1);
+    s_abort = 0;
+    mbar_init(bar(B_QFULL), 1);
+    for (int i = 0; i < KS; ++i) {
+      mbar_init(bar(B_KFULL + i), 1);
+      mbar_init(bar(B_KEMPTY + i), 1 + 256);
+    }
+    for (int i = 0; i < VS; ++i) {
+      mbar_init(bar(B_VFULL + i), 1);
+      mbar_init(bar(B_VEMPTY + i), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar(B_SFULL + x), 1);
+      mbar_init(bar(B_PFULL + x), 128);
+      mbar_init(bar(B_OFULL + x), 1);
+      mbar_init(bar(B_QZ + x), 128);
+    }
     mbar_fence_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmQ);
@@ -129,219 +179,309 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + T;
-  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
   const int Wmax = sW[H - 1];
+  // steps of each query tile and number of key tiles walked (identical in every role)
+  const int dlim = (Wmax + T - 1) / T + 1;  // first tile distance no pair reaches
+  const int nA = min(itA + 1, dlim);
+  const int nB = (itB * T < P.N) ? min(itB + 1, dlim) : 0;
+  const int Tt = max(nB, nA + 1);
+  volatile int* abortp = &s_abort;
+  unsigned int fail_site = 0;
 
-  if (tid == 0) {
-    mbar_expect_tx(bar_q, NB * BLK_BYTES);
-    for (int kb = 0; kb < NB; ++kb) tma_load_3d(sQ + kb * BLK_BYTES, &tmQ, bar_q, kb * 64, it * T, bhq);
-  }
-  bool ok = __syncthreads_and(mbar_wait(bar_q, 0) ? 1 : 0);
-  unsigned int fail_site = ok ? 0u : 1u;
-
-  float m_run = -INFINITY, l_run = 0.f;
-  int zeroed_from = H;  // pairs p >= zeroed_from are zero in the shared copy of Q
-  uint32_t ph_kv = 0, ph_mma = 0;
-  bool first = true;
-  unsigned long long cnt = 0;
-
-  for (int jt = it; jt >= 0 && ok; --jt) {
-    const int dt = it - jt;
-    const int zmin = dt == 0 ? 0 : (dt - 1) * T + 1;
-    const int zmax = (dt + 1) * T - 1;
-    const int p_any = count_ge(sW, H, zmin);
-    const int p_all = count_ge(sW, H, zmax);
-    if (p_any == 0) break;  // no pair reaches this tile, nor any farther one
-    int depth;
-    if (MODE == ATF_MODE_EXACT)
-      depth = p_all;
-    else
-      depth = dt == 0 ? H : min(H, (p_any + 7) / 8 * 8);
-    const int natoms = (depth + 7) / 8;
-    const int ncols_k = MODE == ATF_MODE_EXACT ? 2 * p_any : 2 * depth;
-    const int nkb = (ncols_k + 63) / 64;
-
-    if (MODE == ATF_MODE_EXACT && p_all < zeroed_from) {
-      for (int p = p_all; p < zeroed_from; ++p) {
-        const int col = 2 * p;
-        uint8_t* qa = smem_gen + SM::Q_OFF + (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) + (col & 7) * 2;
-        *reinterpret_cast<uint32_t*>(qa) = 0u;
+  if (warp == 0) {
+    // =============================== TMA producer ===============================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (lane == 0) {
+      mbar_expect_tx(bar(B_QFULL), 2 * SM::TILE);
+      for (int x = 0; x < 2; ++x)
+        for (int kb = 0; kb < NB; ++kb)
+          tma_load_3d(sQ + x * SM::TILE + kb * BLK_BYTES, &tmQ, bar(B_QFULL), kb * 64, (itA + x) * T, bhq);
+      TileSched sc;
+      for (int t = 0; t < Tt; ++t) {
+        const int j = itB - t;
+        const int dnear = max(t - 1, 0);  // the closer user of this key tile
+        sc.advance(sW, H, dnear);
+        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_all, dnear);
+        const int ncols = MODE == ATF_MODE_EXACT ? 2 * (H - sc.r_any) : 2 * depth;
+        const int nkb = max(1, (ncols + 63) / 64);
+        const int ks = t % KS, vs = t % VS;
+        if (!wait_or_abort(bar(B_KEMPTY + ks), ((t / KS) & 1) ^ 1, abortp)) { fail_site = 10; break; }
+        mbar_expect_tx(bar(B_KFULL + ks), nkb * BLK_BYTES);
+        for (int kb = 0; kb < nkb; ++kb)
+          tma_load_3d(sK + ks * SM::TILE + kb * BLK_BYTES, &tmK, bar(B_KFULL + ks), kb * 64, j * T, bhk);
+        if (!wait_or_abort(bar(B_VEMPTY + vs), ((t / VS) & 1) ^ 1, abortp)) { fail_site = 11; break; }
+        mbar_expect_tx(bar(B_VFULL + vs), SM::TILE);
+        for (int kb = 0; kb < NB; ++kb)
+          tma_load_3d(sV + vs * SM::TILE + kb * BLK_BYTES, &tmV, bar(B_VFULL + vs), kb * 64, j * T, bhk);
       }
-      zeroed_from = p_all;
-      fence_proxy_async_smem();
     }
-    if (tid == 0) {
-      mbar_expect_tx(bar_kv, (nkb + NB) * BLK_BYTES);
-      for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sK + kb * BLK_BYTES, &tmK, bar_kv, kb * 64, jt * T, bhk);
-      for (int kb = 0; kb < NB; ++kb) tma_load_3d(sV + kb * BLK_BYTES, &tmV, bar_kv, kb * 64, jt * T, bhk);
-    }
-    __syncthreads();
-    ok = __syncthreads_and(mbar_wait(bar_kv, ph_kv) ? 1 : 0);
-    ph_kv ^= 1;
-    if (!ok) { fail_site = 2; break; }
-
-    // ---- S = Q K^T over the live depth ----
-    if (natoms > 0) {
-      if (tid == 0) {
-        tc_fence_after();
+  } else if (warp == 1) {
+    // =============================== MMA issuer ===============================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (lane == 0) {
+      const uint32_t tS[2] = {tmem_base, tmem_base + T};
+      const uint32_t tO[2] = {tmem_base + 2 * T, tmem_base + 2 * T + D};
+      TileSched sc[2];
+      // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
+      auto issue_qk = [&](int X, int v, int tile) {
+        sc[X].advance(sW, H, v);
+        const int depth = tile_depth<MODE>(H, H - sc[X].r_any, H - sc[X].r_all, v);
+        const int natoms = (depth + 7) / 8;
+        const uint32_t qb = sQ + X * SM::TILE, kb = sK + (tile % KS) * SM::TILE;
         for (int a = 0; a < natoms; ++a) {
           const uint32_t off = (a >> 2) * BLK_BYTES + (a & 3) * 32;
-          tc_mma_ss(tS, make_smem_desc_sw128(sQ + off, 16, 1024), make_smem_desc_sw128(sK + off, 16, 1024), IDESC_QK,
-                    a > 0 ? 1u : 0u);
+          tc_mma_ss(tS[X], make_smem_desc_sw128(qb + off, 16, 1024), make_smem_desc_sw128(kb + off, 16, 1024),
+                    IDESC_QK, a > 0 ? 1u : 0u);
         }
-        tc_commit(bar_mma);
+        tc_commit(bar(B_SFULL + X));
+      };
+      auto issue_pv = [&](int X, int v, int tile) {
+        const uint32_t vb = sV + (tile % VS) * SM::TILE;
+#pragma unroll
+        for (int ks = 0; ks < T / 16; ++ks)
+          tc_mma_ts(tO[X], tS[X] + ks * 8, make_smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), IDESC_PV,
+                    (v == 0 && ks == 0) ? 0u : 1u);
+      };
+      bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
+      if (!ok) fail_site = 20;
+      if (ok && nB > 0) {
+        ok = wait_or_abort(bar(B_KFULL + 0), 0, abortp) && wait_or_abort(bar(B_QZ + 1), 0, abortp);
+        if (ok) {
+          tc_fence_after();
+          issue_qk(1, 0, 0);
+        } else {
+          fail_site = 21;
+        }
       }
-      ok = __syncthreads_and(mbar_wait(bar_mma, ph_mma) ? 1 : 0);
-      ph_mma ^= 1;
-      if (!ok) { fail_site = 3; break; }
-      tc_fence_after();
-    }
-
-    float s[T];
-    if (natoms > 0) {
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + lane_off + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-      tc_wait_ld();
-    } else {
-#pragma unroll
-      for (int c = 0; c < T; ++c) s[c] = 0.f;
-    }
-
-    const int m0 = jt * T;
-    // ---- straddling pairs: add the term only where the distance is inside the pair's window ----
-    if (MODE == ATF_MODE_EXACT) {
-      for (int p = p_all; p < p_any; ++p) {
-        const int wp = sW[H - 1 - p];
-        float q0 = 0.f, q1 = 0.f;
-        if (n < P.N) {
-          const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
-          q0 = bf16lo_to_f32(qq);
-          q1 = bf16hi_to_f32(qq);
+      if (ok) tc_commit(bar(B_KEMPTY + 0));
+      for (int s = 0; s < Tt && ok; ++s) {
+        const bool pvB = s < nB, pvA = s >= 1 && s - 1 < nA;
+        const bool qkB = s + 1 < nB, qkA = s < nA;
+        if (pvB || pvA) ok = ok && wait_or_abort(bar(B_VFULL + s % VS), (s / VS) & 1, abortp);
+        if (qkB || qkA) ok = ok && wait_or_abort(bar(B_KFULL + (s + 1) % KS), ((s + 1) / KS) & 1, abortp);
+        if (!ok) { fail_site = 22; break; }
+        if (pvB) {
+          if (!wait_or_abort(bar(B_PFULL + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
+          tc_fence_after();
+          issue_pv(1, s, s);
         }
-        const int col = 2 * p;
-        const uint8_t* kbase = smem_gen + SM::K_OFF + (col >> 6) * BLK_BYTES + (col & 7) * 2;
-        const int chunk = (col & 63) >> 3;
-        const int zrow = n - m0;  // distance to column 0 of the tile
+        if (qkB) issue_qk(1, s + 1, s + 1);
+        else if (pvB) tc_commit(bar(B_OFULL + 1));
+        if (pvA) {
+          if (!wait_or_abort(bar(B_PFULL + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
+          tc_fence_after();
+          issue_pv(0, s - 1, s);
+        }
+        if (qkA) {
+          if (s == 0 && !wait_or_abort(bar(B_QZ + 0), 0, abortp)) { ok = false; fail_site = 25; break; }
+          tc_fence_after();
+          issue_qk(0, s, s + 1);
+        } else if (pvA) {
+          tc_commit(bar(B_OFULL + 0));
+        }
+        if (s + 1 < Tt) tc_commit(bar(B_KEMPTY + (s + 1) % KS));
+        tc_commit(bar(B_VEMPTY + s % VS));
+      }
+    }
+  } else if (warp >= 4) {
+    // =============================== softmax groups ===============================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int X = warp >= 8 ? 1 : 0;
+    const int row = tid - (X ? 256 : 128);
+    const int itX = X ? itB : itA;
+    const int nX = X ? nB : nA;
+    const int n = itX * T + row;
+    const bool row_ok = n < P.N;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem_base + X * T + lane_off;
+    const uint32_t tO = tmem_base + 2 * T + X * D + lane_off;
+    uint8_t* qrow_base = smem_gen + SM::Q_OFF + X * SM::TILE;
+
+    bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
+    if (!ok) fail_site = 30;
+    TileSched sc;
+    int zeroed_from = H;  // pairs p >= zeroed_from are zero in the shared copy of Q_X
+    auto zero_q_down_to = [&](int p_all) {
+      if (MODE == ATF_MODE_EXACT && p_all < zeroed_from) {
+        for (int p = p_all; p < zeroed_from; ++p) {
+          const int col = 2 * p;
+          *reinterpret_cast<uint32_t*>(qrow_base + (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) +
+                                       (col & 7) * 2) = 0u;
+        }
+        zeroed_from = p_all;
+        fence_proxy_async_smem();
+      }
+    };
+    if (ok) {
+      sc.advance(sW, H, 0);
+      zero_q_down_to(H - sc.r_all);
+      mbar_arrive(bar(B_QZ + X));
+    }
+
+    float m_used = -INFINITY, l_run = 0.f;  // m_used in raw score units
+    unsigned long long cnt = 0;
+
+    for (int t = 0; t < Tt && ok; ++t) {
+      const int v = X ? t : t - 1;  // step of this query tile = its tile distance to key tile t
+      const bool active = v >= 0 && v < nX;
+      const int ks = t % KS;
+      if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
+      if (!active) {
+        mbar_arrive(bar(B_KEMPTY + ks));
+        continue;
+      }
+      const int dt = v;
+      const int zmax = (dt + 1) * T - 1;
+      const int p_any = H - sc.r_any, p_all = H - sc.r_all;  // cursors already at dt
+      const int depth = tile_depth<MODE>(H, p_any, p_all, dt);
+      const int natoms = (depth + 7) / 8;
+      if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
+      tc_fence_after();
+
+      float s[T];
+      if (natoms > 0) {
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int c = 0; c < T; ++c) s[c] = 0.f;
+      }
+      const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
+
+      // ---- straddling pairs: add the term only where the distance is inside the pair's window ----
+      if (MODE == ATF_MODE_EXACT) {
+        for (int p = p_all; p < p_any; ++p) {
+          const int wp = sW[H - 1 - p];
+          float q0 = 0.f, q1 = 0.f;
+          if (row_ok) {
+            const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
+            q0 = bf16lo_to_f32(qq);
+            q1 = bf16hi_to_f32(qq);
+          }
+          const int col = 2 * p;
+          const uint8_t* kbase = smem_gen + SM::K_OFF + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+          const int chunk = (col & 63) >> 3;
+#pragma unroll
+          for (int c = 0; c < T; ++c) {
+            const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
+            const float add = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
+            s[c] += (zrow - c <= wp) ? add : 0.f;
+          }
+          if (COUNT && row_ok) {
+            const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
+            cnt += (unsigned long long)max(0, hi - lo + 1);
+          }
+        }
+      }
+      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
+      if (COUNT && row_ok) {
+        const int ncols = dt == 0 ? row + 1 : T;
+        cnt += (unsigned long long)depth * (unsigned long long)ncols;
+      }
+
+      // ---- causal mask, dropped keys (exact mode: per cell), running max ----
+      const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
+      float mx = -INFINITY;
+      if (dt == 0 || zmax > zdrop) {
 #pragma unroll
         for (int c = 0; c < T; ++c) {
-          const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
-          const float add = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
-          s[c] += (zrow - c <= wp) ? add : 0.f;
+          const int z = zrow - c;
+          s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
+          mx = fmaxf(mx, s[c]);
         }
-        if (COUNT && n < P.N) {
-          const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
-          cnt += (unsigned long long)max(0, hi - lo + 1);
-        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < T; ++c) mx = fmaxf(mx, s[c]);
       }
-    }
-    if (COUNT && n < P.N) {
-      const int ncols = dt == 0 ? row + 1 : T;
-      cnt += (unsigned long long)depth * (unsigned long long)ncols;
-    }
-
-    // ---- scale, causal mask, drop keys no pair reaches (exact mode: per cell; coarse mode
-    //      decides per tile, which the loop exit above already did), online softmax ----
-    const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
-    const bool need_mask = (dt == 0) || (zmax > zdrop);
-    float mx = -INFINITY;
-    if (need_mask) {
-      const int zrow = n - m0;
+      // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
+      float scale_o = 1.f;
+      bool moved = false;
+      if (v == 0) {
+        m_used = mx;  // finite: the diagonal cell of every row is live
+      } else if ((mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD) {
+        scale_o = exp2f((m_used - mx) * kScaleLog2);
+        m_used = mx;
+        moved = true;
+      }
+      const bool any_moved = __any_sync(0xffffffffu, moved);
+      const float neg_m = -m_used * kScaleLog2;
+      float psum = 0.f;
 #pragma unroll
       for (int c = 0; c < T; ++c) {
-        const int z = zrow - c;
-        s[c] = (z >= 0 && z <= zdrop) ? s[c] * kScaleLog2 : -INFINITY;
-        mx = fmaxf(mx, s[c]);
+        s[c] = exp2f(fmaf(s[c], kScaleLog2, neg_m));
+        psum += s[c];
       }
-    } else {
-#pragma unroll
-      for (int c = 0; c < T; ++c) {
-        s[c] *= kScaleLog2;
-        mx = fmaxf(mx, s[c]);
-      }
-    }
-    const float m_new = fmaxf(m_run, mx);
-    const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = exp2f(m_run - m_safe);
-    m_run = m_new;
-    float psum = 0.f;
-#pragma unroll
-    for (int c = 0; c < T; ++c) {
-      s[c] = exp2f(s[c] - m_safe);
-      psum += s[c];
-    }
-    l_run = l_run * alpha + psum;
+      l_run = l_run * scale_o + psum;
 
-    // ---- P (bf16) into tensor memory, over the first 64 columns of S: column c of a lane
-    //      holds keys 2c (low half) and 2c+1 (high half) of that query row ----
-    {
-      uint32_t pk[64];
+      // ---- P (bf16) over the first 64 columns of S: column c holds keys 2c and 2c+1 ----
+      {
+        uint32_t pk[64];
 #pragma unroll
-      for (int c = 0; c < 64; ++c) pk[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
-      tc_st32(tS + lane_off, pk);
-      tc_st32(tS + lane_off + 32, pk + 32);
+        for (int c = 0; c < 64; ++c) pk[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
+        tc_st32(tS, pk);
+        tc_st32(tS + 32, pk + 32);
+      }
+      if (any_moved) {
+#pragma unroll
+        for (int q4 = 0; q4 < D / 32; ++q4) {
+          uint32_t o[32];
+          tc_ld32(tO + q4 * 32, o);
+          tc_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
+          tc_st32(tO + q4 * 32, o);
+        }
+      }
+      // zero the Q columns that stop being live everywhere at the next step
+      if (v + 1 < nX) {
+        sc.advance(sW, H, dt + 1);
+        zero_q_down_to(H - sc.r_all);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(B_PFULL + X));
     }
-    // ---- rescale O ----
-    if (!first) {
+
+    if (ok && nX > 0) {
+      if (!wait_or_abort(bar(B_OFULL + X), 0, abortp)) {
+        ok = false;
+        fail_site = 33;
+      }
+    }
+    if (ok && nX > 0) {
+      tc_fence_after();
+      const float inv = 1.f / l_run;
+      __nv_bfloat16* orow = P.O + ((int64_t)bhq * P.N + n) * D;
 #pragma unroll
       for (int q4 = 0; q4 < D / 32; ++q4) {
         uint32_t o[32];
-        tc_ld32(tO + lane_off + q4 * 32, o);
+        tc_ld32(tO + q4 * 32, o);
         tc_wait_ld();
+        if (row_ok) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-        tc_st32(tO + lane_off + q4 * 32, o);
-      }
-    }
-    tc_wait_st();
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- O += P V ----
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < T / 16; ++ks) {
-        const uint64_t db = make_smem_desc_sw128(sV + ks * 2048, BLK_BYTES, 1024);
-        tc_mma_ts(tO, tS + ks * 8, db, IDESC_PV, (first && ks == 0) ? 0u : 1u);
-      }
-      tc_commit(bar_mma);
-    }
-    ok = __syncthreads_and(mbar_wait(bar_mma, ph_mma) ? 1 : 0);
-    ph_mma ^= 1;
-    if (!ok) { fail_site = 4; break; }
-    tc_fence_after();
-    first = false;
-  }
-
-  if (ok) {
-    // ---- epilogue: O / l, LSE ----
-    const float inv = 1.f / l_run;
-    __nv_bfloat16* orow = P.O + ((int64_t)bhq * P.N + n) * D;
-#pragma unroll
-    for (int q4 = 0; q4 < D / 32; ++q4) {
-      uint32_t o[32];
-      tc_ld32(tO + lane_off + q4 * 32, o);
-      tc_wait_ld();
-      if (n < P.N) {
-#pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          uint4 v;
-          v.x = pack_bf16x2(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
-          v.y = pack_bf16x2(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-          v.z = pack_bf16x2(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-          v.w = pack_bf16x2(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-          *reinterpret_cast<uint4*>(orow + q4 * 32 + e) = v;
+          for (int e = 0; e < 32; e += 8) {
+            uint4 v4;
+            v4.x = pack_bf16x2(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
+            v4.y = pack_bf16x2(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+            v4.z = pack_bf16x2(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+            v4.w = pack_bf16x2(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + q4 * 32 + e) = v4;
+          }
         }
       }
-    }
-    if (P.LSE && n < P.N) P.LSE[(int64_t)bhq * P.N + n] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-    if (COUNT) {
+      if (P.LSE && row_ok) P.LSE[(int64_t)bhq * P.N + n] = (m_used * kScaleLog2 + log2f(l_run)) * 0.6931471805599453f;
+      if (COUNT) {
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-      if ((tid & 31) == 0 && cnt) atomicAdd(P.kept + bhq, cnt);
+        for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+        if (lane == 0 && cnt) atomicAdd(P.kept + bhq, cnt);
+      }
     }
-  } else if (tid == 0) {
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  }
+
+  if (fail_site) {
     atomicExch(P.status, 1u);
     atomicExch(P.status + 1, fail_site);
   }
@@ -384,14 +524,14 @@ atf_status make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N
 template <int D>
 atf_status launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& P,
                           const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
-  const int nqt = (P.N + T - 1) / T;
-  dim3 grid(nqt, P.Hq, B);
+  const int npt = (P.N + 2 * T - 1) / (2 * T);
+  dim3 grid(npt, P.Hq, B);
   const int smem = PrefillSmem<D>::DYN_BYTES;
 #define ATF_PF_LAUNCH(MODE_, COUNT_)                                                                        \
   do {                                                                                                      \
     auto kern = atf_prefill_kernel<D, MODE_, COUNT_>;                                                       \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));          \
-    kern<<<grid, 128, smem, s>>>(tq, tk, tv, P, t);                                                         \
+    kern<<<grid, PF_THREADS, smem, s>>>(tq, tk, tv, P, t);                                                         \
   } while (0)
   if (mode == ATF_MODE_EXACT) {
     if (count) ATF_PF_LAUNCH(ATF_MODE_EXACT, true); else ATF_PF_LAUNCH(ATF_MODE_EXACT, false);
@@ -424,7 +564,7 @@ extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V
   if (B < 1 || Hq < 1 || Hkv < 1 || N < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: bad shape");
   if (Hq % Hkv) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: Hq must be a multiple of Hkv");
   if (!causal) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: only causal attention is defined (distance z = n - m >= 0)");
-  if (N >= (1ll << 31) - 2 * T) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: N too large");
+  if (N >= (1ll << 31) - 4 * T) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: N too large");
   if (Hq > 65535 || B > 65535) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: B and Hq must be <= 65535");
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O) & 15)
     return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: pointers must be 16-byte aligned");
