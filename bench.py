@@ -174,10 +174,11 @@ def run_ours(args):
         atf.atf_rope(Qg, theta)
         atf.atf_rope(Kg, theta)
         e[2].record()
-        atf.atf_prefill(Qg, Kg, V, table=W, O=O, LSE=LSE)
+        Wuse = None if args.full_attention else W
+        atf.atf_prefill(Qg, Kg, V, table=Wuse, O=O, LSE=LSE)
         e[3].record()
         qd.copy_(Qg[:, :, -1])
-        atf.atf_decode(qd, Kg, V, table=W, O=Od)
+        atf.atf_decode(qd, Kg, V, table=Wuse, O=Od)
         e[4].record()
         if timed:
             torch.cuda.synchronize()
@@ -367,6 +368,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="llama3b-128k")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--full-attention", action="store_true",
+                    help="run the step with table = NULL (the library's own k = infinity mode)")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only the warm-up and timed steps (for ncu captures); prints a short line")
     args = ap.parse_args()

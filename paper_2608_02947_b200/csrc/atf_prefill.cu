@@ -86,18 +86,31 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
 // span distances [zmin, zmax].  w[] is non-decreasing, so the pairs reaching a distance z are
 // r >= r0(z), and r0 only grows with dt: the cursors are advanced, never rewound.
 struct TileSched {
-  int r_any = 0, r_all = 0;  // first pair live in some cell / in every cell
+  // first pair live in some cell / in most cells (window reaches the tile's central distance)
+  // / in every cell of the tile
+  int r_any = 0, r_mid = 0, r_all = 0;
   __device__ __forceinline__ void advance(const int* w, int H, int dt) {
     const int zmin = dt == 0 ? 0 : (dt - 1) * T + 1;
+    const int zmid = dt == 0 ? T / 2 : dt * T;
     const int zmax = (dt + 1) * T - 1;
     while (r_any < H && w[r_any] < zmin) ++r_any;
+    while (r_mid < H && w[r_mid] < zmid) ++r_mid;
     while (r_all < H && w[r_all] < zmax) ++r_all;
   }
 };
+// Pairs contracted by the MMA for a tile.  Exact mode: the pairs live in most cells (the few
+// cells where a pair of those is dead are subtracted afterwards; pairs live in only a minority
+// of the cells are left out and added where live).  Coarse mode: pairs live anywhere in the
+// tile, rounded up to a group of 8; everything on the diagonal tile.
 template <int MODE>
-__device__ __forceinline__ int tile_depth(int H, int p_any, int p_all, int dt) {
-  if (MODE == ATF_MODE_EXACT) return p_all;
+__device__ __forceinline__ int tile_depth(int H, int p_any, int p_mid, int dt) {
+  if (MODE == ATF_MODE_EXACT) return p_mid;
   return dt == 0 ? H : min(H, (p_any + 7) / 8 * 8);
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 // Bounded wait that also gives up as soon as another role of the CTA has given up.
@@ -201,7 +214,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const int j = itB - t;
         const int dnear = max(t - 1, 0);  // the closer user of this key tile
         sc.advance(sW, H, dnear);
-        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_all, dnear);
+        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, dnear);
         const int ncols = MODE == ATF_MODE_EXACT ? 2 * (H - sc.r_any) : 2 * depth;
         const int nkb = max(1, (ncols + 63) / 64);
         const int ks = t % KS, vs = t % VS;
@@ -225,7 +238,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
       auto issue_qk = [&](int X, int v, int tile) {
         sc[X].advance(sW, H, v);
-        const int depth = tile_depth<MODE>(H, H - sc[X].r_any, H - sc[X].r_all, v);
+        const int depth = tile_depth<MODE>(H, H - sc[X].r_any, H - sc[X].r_mid, v);
         const int natoms = (depth + 7) / 8;
         const uint32_t qb = sQ + X * SM::TILE, kb = sK + (tile % KS) * SM::TILE;
         for (int a = 0; a < natoms; ++a) {
@@ -301,20 +314,20 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     if (!ok) fail_site = 30;
     TileSched sc;
     int zeroed_from = H;  // pairs p >= zeroed_from are zero in the shared copy of Q_X
-    auto zero_q_down_to = [&](int p_all) {
-      if (MODE == ATF_MODE_EXACT && p_all < zeroed_from) {
-        for (int p = p_all; p < zeroed_from; ++p) {
+    auto zero_q_down_to = [&](int p_keep) {
+      if (MODE == ATF_MODE_EXACT && p_keep < zeroed_from) {
+        for (int p = p_keep; p < zeroed_from; ++p) {
           const int col = 2 * p;
           *reinterpret_cast<uint32_t*>(qrow_base + (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) +
                                        (col & 7) * 2) = 0u;
         }
-        zeroed_from = p_all;
+        zeroed_from = p_keep;
         fence_proxy_async_smem();
       }
     };
     if (ok) {
       sc.advance(sW, H, 0);
-      zero_q_down_to(H - sc.r_all);
+      zero_q_down_to(H - sc.r_mid);
       mbar_arrive(bar(B_QZ + X));
     }
 
@@ -332,8 +345,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
       const int dt = v;
       const int zmax = (dt + 1) * T - 1;
-      const int p_any = H - sc.r_any, p_all = H - sc.r_all;  // cursors already at dt
-      const int depth = tile_depth<MODE>(H, p_any, p_all, dt);
+      const int p_any = H - sc.r_any, p_mid = H - sc.r_mid, p_all = H - sc.r_all;  // cursors already at dt
+      const int depth = tile_depth<MODE>(H, p_any, p_mid, dt);
       const int natoms = (depth + 7) / 8;
       if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
       tc_fence_after();
@@ -349,24 +362,42 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
 
-      // ---- straddling pairs: add the term only where the distance is inside the pair's window ----
+      // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
+      //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
+      //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
+      //      no row of this warp has such a cell in it. ----
       if (MODE == ATF_MODE_EXACT) {
+        const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
         for (int p = p_all; p < p_any; ++p) {
           const int wp = sW[H - 1 - p];
+          const bool subtract = p < p_mid;
           float q0 = 0.f, q1 = 0.f;
           if (row_ok) {
             const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
             q0 = bf16lo_to_f32(qq);
             q1 = bf16hi_to_f32(qq);
           }
+          if (subtract) {
+            q0 = -q0;
+            q1 = -q1;
+          }
           const int col = 2 * p;
           const uint8_t* kbase = smem_gen + SM::K_OFF + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
           const int chunk = (col & 63) >> 3;
 #pragma unroll
-          for (int c = 0; c < T; ++c) {
-            const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
-            const float add = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
-            s[c] += (zrow - c <= wp) ? add : 0.f;
+          for (int q4 = 0; q4 < 4; ++q4) {
+            // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
+            const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
+            if (touched) {
+#pragma unroll
+              for (int cc = 0; cc < 32; ++cc) {
+                const int c = q4 * 32 + cc;
+                const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
+                const float term = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
+                const bool inside = zrow - c <= wp;
+                s[c] += (inside != subtract) ? term : 0.f;
+              }
+            }
           }
           if (COUNT && row_ok) {
             const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
@@ -377,22 +408,27 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
       if (COUNT && row_ok) {
         const int ncols = dt == 0 ? row + 1 : T;
-        cnt += (unsigned long long)depth * (unsigned long long)ncols;
+        cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
       }
 
       // ---- causal mask, dropped keys (exact mode: per cell), running max ----
       const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
-      float mx = -INFINITY;
       if (dt == 0 || zmax > zdrop) {
 #pragma unroll
         for (int c = 0; c < T; ++c) {
           const int z = zrow - c;
           s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
-          mx = fmaxf(mx, s[c]);
         }
-      } else {
+      }
+      float mx;
+      {
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < T; ++c) mx = fmaxf(mx, s[c]);
+        for (int c = 0; c < T; c += 8) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
       // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
       float scale_o = 1.f;
@@ -400,17 +436,27 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       if (v == 0) {
         m_used = mx;  // finite: the diagonal cell of every row is live
       } else if ((mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD) {
-        scale_o = exp2f((m_used - mx) * kScaleLog2);
+        scale_o = ex2_approx((m_used - mx) * kScaleLog2);
         m_used = mx;
         moved = true;
       }
       const bool any_moved = __any_sync(0xffffffffu, moved);
       const float neg_m = -m_used * kScaleLog2;
-      float psum = 0.f;
+      float psum;
+      {
+        const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
+        float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-      for (int c = 0; c < T; ++c) {
-        s[c] = exp2f(fmaf(s[c], kScaleLog2, neg_m));
-        psum += s[c];
+        for (int c = 0; c < T; c += 2) {
+          float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
+          x.x = ex2_approx(x.x);
+          x.y = ex2_approx(x.y);
+          s[c] = x.x;
+          s[c + 1] = x.y;
+          acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
+        }
+        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+        psum = (a01.x + a01.y) + (a23.x + a23.y);
       }
       l_run = l_run * scale_o + psum;
 
@@ -436,7 +482,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // zero the Q columns that stop being live everywhere at the next step
       if (v + 1 < nX) {
         sc.advance(sW, H, dt + 1);
-        zero_q_down_to(H - sc.r_all);
+        zero_q_down_to(H - sc.r_mid);
       }
       tc_wait_st();
       tc_fence_before();
