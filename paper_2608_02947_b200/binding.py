@@ -29,7 +29,8 @@ class _Opts(C.Structure):
 
 
 def lib_path():
-    return os.path.join(_HERE, "libatflash.so")
+    """Path of the shared library (ATFLASH_LIB overrides the in-tree build, e.g. to compare builds)."""
+    return os.environ.get("ATFLASH_LIB") or os.path.join(_HERE, "libatflash.so")
 
 
 _lib = None

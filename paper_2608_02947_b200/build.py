@@ -21,7 +21,8 @@ LIB = os.path.join(HERE, "libatflash.so")
 SOURCES = ["atf_host.cu", "atf_rope.cu", "atf_decode.cu", "atf_prefill.cu"]
 HEADERS = [os.path.join(CSRC, "atf_common.cuh"), os.path.join(ROOT, "include", "atflash.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+EXTRA = os.environ.get("ATF_NVCC_EXTRA", "").split()
+FLAGS = EXTRA + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 

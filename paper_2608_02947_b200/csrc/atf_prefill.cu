@@ -28,6 +28,8 @@
 // Coarse mode: depth = pairs live in any cell of the tile, rounded up to 8; diagonal tile full.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "atf_common.cuh"
 
 namespace {
@@ -36,9 +38,27 @@ constexpr int T = 128;              // query rows per tile and key columns per t
 constexpr int BLK_BYTES = T * 128;  // one [128 x 64] bf16 block, 128-byte rows
 constexpr int KS = 2, VS = 2;       // ring depths
 constexpr int PF_THREADS = 384;
+// Register budget.  The kernel is compiled for 168 registers per thread (65536 / 384, rounded
+// down to a multiple of 8), i.e. 64512 in use at launch.  The producer/MMA warpgroup then
+// shrinks to 72 and the two softmax warpgroups grow to 216: 128*72 + 256*216 = 64512.  The
+// total after the change must not exceed the total at launch, or the growing warps wait for
+// registers that never come.
+static_assert(128 * 72 + 256 * 216 <= PF_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag behind
 
+// Optional timeline tracing (compile with -DATF_TRACE): block (0,0,0) stamps %clock64 at a few
+// events per step into the first words of the repacked-K scratch tail.  Off in normal builds.
+#ifdef ATF_TRACE
+#define ATF_STAMP(slot, step) do { if (blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && (step) < 64) \
+    P.trace[(slot) * 64 + (step)] = clock64(); } while (0)
+#else
+#define ATF_STAMP(slot, step) do { } while (0)
+#endif
+#ifndef ATF_TRACE_BLOCK
+#define ATF_TRACE_BLOCK 0
+#endif
 struct PrefillParams {
+  long long* trace;
   const __nv_bfloat16* Qp;  // pair-interleaved copy of Q, [B*Hq, N, D]
   __nv_bfloat16* O;
   float* LSE;
@@ -106,6 +126,29 @@ template <int MODE>
 __device__ __forceinline__ int tile_depth(int H, int p_any, int p_mid, int dt) {
   if (MODE == ATF_MODE_EXACT) return p_mid;
   return dt == 0 ? H : min(H, (p_any + 7) / 8 * 8);
+}
+// 2^x for a pair of values on the FMA pipe (x <= ~8; anything below -126, -inf included, gives
+// ~1e-38): round x to the nearest integer n with the 1.5*2^23 trick, evaluate a cubic minimax
+// of 2^f on f = x - n in [-0.5, 0.5] (relative error < 8e-5, below the bf16 rounding of P),
+// and add n to the exponent field.
+#ifndef ATF_POLY_OF_4
+#define ATF_POLY_OF_4 2
+#endif
+constexpr int POLY_OF_4 = ATF_POLY_OF_4;  // of every 4 packed pairs, this many take the polynomial, the rest MUFU
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 magic = make_float2(12582912.f, 12582912.f);
+  const float2 t = __fadd2_rn(x, magic);
+  const float2 nf = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __fadd2_rn(x, make_float2(-nf.x, -nf.y));
+  float2 p = __ffma2_rn(make_float2(0.05520550534f, 0.05520550534f), f, make_float2(0.24261397123f, 0.24261397123f));
+  p = __ffma2_rn(p, f, make_float2(0.69325476885f, 0.69325476885f));
+  p = __ffma2_rn(p, f, make_float2(0.99992769957f, 0.99992769957f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return r;
 }
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -203,7 +246,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   if (warp == 0) {
     // =============================== TMA producer ===============================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
       mbar_expect_tx(bar(B_QFULL), 2 * SM::TILE);
       for (int x = 0; x < 2; ++x)
@@ -230,30 +273,38 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
   } else if (warp == 1) {
     // =============================== MMA issuer ===============================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
-      const uint32_t tS[2] = {tmem_base, tmem_base + T};
-      const uint32_t tO[2] = {tmem_base + 2 * T, tmem_base + 2 * T + D};
-      TileSched sc[2];
+      static_assert(KS == 2 && VS == 2, "stage selection below assumes two-stage rings");
+      TileSched scA, scB;
+      // Descriptors are built once; an MMA step only adds a constant to the start-address field
+      // (16-byte units): K-major operands advance 32 bytes per 16-column step inside a
+      // 64-column block and one block per four steps; V advances 16 key rows (2048 bytes).
+      const uint64_t dQ0 = make_smem_desc_sw128(sQ, 16, 1024), dQ1 = make_smem_desc_sw128(sQ + SM::TILE, 16, 1024);
+      const uint64_t dK0 = make_smem_desc_sw128(sK, 16, 1024), dK1 = make_smem_desc_sw128(sK + SM::TILE, 16, 1024);
+      const uint64_t dV0 = make_smem_desc_sw128(sV, BLK_BYTES, 1024),
+                     dV1 = make_smem_desc_sw128(sV + SM::TILE, BLK_BYTES, 1024);
       // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
       auto issue_qk = [&](int X, int v, int tile) {
-        sc[X].advance(sW, H, v);
-        const int depth = tile_depth<MODE>(H, H - sc[X].r_any, H - sc[X].r_mid, v);
+        TileSched& sc = X ? scB : scA;
+        sc.advance(sW, H, v);
+        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, v);
         const int natoms = (depth + 7) / 8;
-        const uint32_t qb = sQ + X * SM::TILE, kb = sK + (tile % KS) * SM::TILE;
-        for (int a = 0; a < natoms; ++a) {
-          const uint32_t off = (a >> 2) * BLK_BYTES + (a & 3) * 32;
-          tc_mma_ss(tS[X], make_smem_desc_sw128(qb + off, 16, 1024), make_smem_desc_sw128(kb + off, 16, 1024),
-                    IDESC_QK, a > 0 ? 1u : 0u);
+        const uint64_t q0 = X ? dQ1 : dQ0, k0 = (tile & 1) ? dK1 : dK0;
+        const uint32_t d = tmem_base + X * T;
+#pragma unroll
+        for (int a = 0; a < D / 16; ++a) {
+          const uint64_t off = (uint64_t)(((a >> 2) * BLK_BYTES + (a & 3) * 32) >> 4);
+          if (a < natoms) tc_mma_ss(d, q0 + off, k0 + off, IDESC_QK, a > 0 ? 1u : 0u);
         }
         tc_commit(bar(B_SFULL + X));
       };
       auto issue_pv = [&](int X, int v, int tile) {
-        const uint32_t vb = sV + (tile % VS) * SM::TILE;
+        const uint64_t v0 = (tile & 1) ? dV1 : dV0;
+        const uint32_t d = tmem_base + 2 * T + X * D, p = tmem_base + X * T;
+        tc_mma_ts(d, p, v0, IDESC_PV, v == 0 ? 0u : 1u);
 #pragma unroll
-        for (int ks = 0; ks < T / 16; ++ks)
-          tc_mma_ts(tO[X], tS[X] + ks * 8, make_smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), IDESC_PV,
-                    (v == 0 && ks == 0) ? 0u : 1u);
+        for (int ks = 1; ks < T / 16; ++ks) tc_mma_ts(d, p + ks * 8, v0 + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
       };
       bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
       if (!ok) fail_site = 20;
@@ -276,13 +327,17 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (pvB) {
           if (!wait_or_abort(bar(B_PFULL + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
           tc_fence_after();
+          ATF_STAMP(10, s);
           issue_pv(1, s, s);
+          ATF_STAMP(11, s);
         }
         if (qkB) issue_qk(1, s + 1, s + 1);
         else if (pvB) tc_commit(bar(B_OFULL + 1));
+        ATF_STAMP(12, s);
         if (pvA) {
           if (!wait_or_abort(bar(B_PFULL + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
           tc_fence_after();
+          ATF_STAMP(13, s);
           issue_pv(0, s - 1, s);
         }
         if (qkA) {
@@ -292,13 +347,14 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         } else if (pvA) {
           tc_commit(bar(B_OFULL + 0));
         }
+        ATF_STAMP(14, s);
         if (s + 1 < Tt) tc_commit(bar(B_KEMPTY + (s + 1) % KS));
         tc_commit(bar(B_VEMPTY + s % VS));
       }
     }
   } else if (warp >= 4) {
     // =============================== softmax groups ===============================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int X = warp >= 8 ? 1 : 0;
     const int row = tid - (X ? 256 : 128);
     const int itX = X ? itB : itA;
@@ -350,125 +406,115 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int natoms = (depth + 7) / 8;
       if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
       tc_fence_after();
+      if (row == 0) ATF_STAMP(0 + 5 * X, v);
 
-      float s[T];
-      if (natoms > 0) {
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-        tc_wait_ld();
-      } else {
-#pragma unroll
-        for (int c = 0; c < T; ++c) s[c] = 0.f;
-      }
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
-
-      // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
-      //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
-      //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
-      //      no row of this warp has such a cell in it. ----
-      if (MODE == ATF_MODE_EXACT) {
-        const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
-        for (int p = p_all; p < p_any; ++p) {
-          const int wp = sW[H - 1 - p];
-          const bool subtract = p < p_mid;
-          float q0 = 0.f, q1 = 0.f;
-          if (row_ok) {
-            const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
-            q0 = bf16lo_to_f32(qq);
-            q1 = bf16hi_to_f32(qq);
-          }
-          if (subtract) {
-            q0 = -q0;
-            q1 = -q1;
-          }
-          const int col = 2 * p;
-          const uint8_t* kbase = smem_gen + SM::K_OFF + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
-          const int chunk = (col & 63) >> 3;
+      const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
+      float s[T];
+      uint32_t pk[T / 2];
+      float psum;
+      // One pass normally.  The exponentials are taken against the reference maximum carried
+      // over from earlier tiles, so they do not wait for this tile's row maximum; if some row's
+      // maximum turns out to lead the reference by more than the threshold, the reference
+      // moves, O and l are rescaled, and the pass is repeated (rare after the first tiles).
+#pragma unroll 1
+      for (int pass = 0;; ++pass) {
+        if (natoms > 0) {
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
-            const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
-            if (touched) {
+          for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+          tc_wait_ld();
+        } else {
 #pragma unroll
-              for (int cc = 0; cc < 32; ++cc) {
-                const int c = q4 * 32 + cc;
-                const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
-                const float term = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
-                const bool inside = zrow - c <= wp;
-                s[c] += (inside != subtract) ? term : 0.f;
+          for (int c = 0; c < T; ++c) s[c] = 0.f;
+        }
+        if (row == 0) ATF_STAMP(1 + 5 * X, v);
+        // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
+        //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
+        //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
+        //      no row of this warp has such a cell in it. ----
+        if (MODE == ATF_MODE_EXACT) {
+          const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
+          for (int p = p_all; p < p_any; ++p) {
+            const int wp = sW[H - 1 - p];
+            const bool subtract = p < p_mid;
+            float q0 = 0.f, q1 = 0.f;
+            if (row_ok) {
+              const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
+              q0 = bf16lo_to_f32(qq);
+              q1 = bf16hi_to_f32(qq);
+            }
+            if (subtract) {
+              q0 = -q0;
+              q1 = -q1;
+            }
+            const int col = 2 * p;
+            const uint8_t* kbase = smem_gen + SM::K_OFF + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+            const int chunk = (col & 63) >> 3;
+  #pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
+              const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
+              if (touched) {
+  #pragma unroll
+                for (int cc = 0; cc < 32; ++cc) {
+                  const int c = q4 * 32 + cc;
+                  const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
+                  const float term = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
+                  const bool inside = zrow - c <= wp;
+                  s[c] += (inside != subtract) ? term : 0.f;
+                }
               }
             }
           }
-          if (COUNT && row_ok) {
-            const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
-            cnt += (unsigned long long)max(0, hi - lo + 1);
+        }
+
+        // ---- causal mask, dropped keys (exact mode: per cell) ----
+        if (dt == 0 || zmax > zdrop) {
+#pragma unroll
+          for (int c = 0; c < T; ++c) {
+            const int z = zrow - c;
+            s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
           }
         }
-      }
-      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
-      if (COUNT && row_ok) {
-        const int ncols = dt == 0 ? row + 1 : T;
-        cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
-      }
-
-      // ---- causal mask, dropped keys (exact mode: per cell), running max ----
-      const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
-      if (dt == 0 || zmax > zdrop) {
+        float mx;
+        {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < T; ++c) {
-          const int z = zrow - c;
-          s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
+          for (int c = 0; c < T; c += 8) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+          }
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
-      }
-      float mx;
-      {
-        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (v == 0 && pass == 0) m_used = mx;  // finite: the diagonal cell of every row is live
+        const float neg_m = -m_used * kScaleLog2;
+        {
+          const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
+          float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int c = 0; c < T; c += 8) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+          for (int c = 0; c < T; c += 2) {
+            float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
+            if (((c >> 1) & 3) < POLY_OF_4) {
+              x = exp2_poly2(x);
+            } else {
+              x.x = ex2_approx(x.x);
+              x.y = ex2_approx(x.y);
+            }
+            acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
+            pk[c >> 1] = pack_bf16x2(x.x, x.y);
+          }
+          const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+          psum = (a01.x + a01.y) + (a23.x + a23.y);
         }
-        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-      }
-      // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
-      float scale_o = 1.f;
-      bool moved = false;
-      if (v == 0) {
-        m_used = mx;  // finite: the diagonal cell of every row is live
-      } else if ((mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD) {
-        scale_o = ex2_approx((m_used - mx) * kScaleLog2);
-        m_used = mx;
-        moved = true;
-      }
-      const bool any_moved = __any_sync(0xffffffffu, moved);
-      const float neg_m = -m_used * kScaleLog2;
-      float psum;
-      {
-        const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
-        float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-        for (int c = 0; c < T; c += 2) {
-          float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
-          x.x = ex2_approx(x.x);
-          x.y = ex2_approx(x.y);
-          s[c] = x.x;
-          s[c + 1] = x.y;
-          acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
+        const bool lag = (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD;
+        if (!__any_sync(0xffffffffu, lag)) break;
+        // move the reference maximum of the lagging rows, rescale their O and l, redo the pass
+        float scale_o = 1.f;
+        if (lag) {
+          scale_o = ex2_approx((m_used - mx) * kScaleLog2);
+          m_used = mx;
+          l_run *= scale_o;
         }
-        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
-        psum = (a01.x + a01.y) + (a23.x + a23.y);
-      }
-      l_run = l_run * scale_o + psum;
-
-      // ---- P (bf16) over the first 64 columns of S: column c holds keys 2c and 2c+1 ----
-      {
-        uint32_t pk[64];
-#pragma unroll
-        for (int c = 0; c < 64; ++c) pk[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
-        tc_st32(tS, pk);
-        tc_st32(tS + 32, pk + 32);
-      }
-      if (any_moved) {
 #pragma unroll
         for (int q4 = 0; q4 < D / 32; ++q4) {
           uint32_t o[32];
@@ -478,14 +524,34 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
           tc_st32(tO + q4 * 32, o);
         }
+        tc_wait_st();
       }
-      // zero the Q columns that stop being live everywhere at the next step
+      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
+      if (row == 0) ATF_STAMP(2 + 5 * X, v);
+      l_run += psum;
+      if (COUNT && row_ok) {
+        const int ncols = dt == 0 ? row + 1 : T;
+        cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
+        if (MODE == ATF_MODE_EXACT) {
+          for (int p = p_all; p < p_any; ++p) {
+            const int wp = sW[H - 1 - p];
+            const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
+            cnt += (unsigned long long)max(0, hi - lo + 1);
+          }
+        }
+      }
+
+      // ---- P (bf16) over the first 64 columns of S: column c holds keys 2c and 2c+1 ----
+      tc_st32(tS, pk);
+      tc_st32(tS + 32, pk + 32);
+      // zero the Q columns that stop being live in most cells at the next step
       if (v + 1 < nX) {
         sc.advance(sW, H, dt + 1);
         zero_q_down_to(H - sc.r_mid);
       }
       tc_wait_st();
       tc_fence_before();
+      if (row == 0) ATF_STAMP(3 + 5 * X, v);
       mbar_arrive(bar(B_PFULL + X));
     }
 
@@ -524,7 +590,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
   } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   }
 
   if (fail_site) {
@@ -598,6 +664,16 @@ size_t repack_bytes(int B, int H, int64_t N, int d) {
 
 atf_status atf_validate_table(const char* who, const int64_t* table, int d, int64_t N, AtfTable* out);
 
+// With -DATF_TRACE the caller passes a device buffer address for the timeline in ATF_TRACE_PTR.
+static void* getenv_trace_ptr() {
+#ifdef ATF_TRACE
+  const char* e = getenv("ATF_TRACE_PTR");
+  return e ? (void*)strtoull(e, nullptr, 0) : nullptr;
+#else
+  return nullptr;
+#endif
+}
+
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d) {
   return ATF_WS_HEADER + repack_bytes(B, Hq, N, d) + repack_bytes(B, Hkv, N, d);
 }
@@ -647,6 +723,7 @@ extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V
   if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
 
   PrefillParams P;
+  P.trace = (long long*)getenv_trace_ptr();
   P.Qp = Qp;
   P.O = (__nv_bfloat16*)O;
   P.LSE = LSE;
