@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     ATF_MODE_COARSE,
     ATF_MODE_EXACT,
     AtfError,
+    WindowTable,
     atf_decode,
     atf_prefill,
     atf_rope,

@@ -99,14 +99,22 @@ def _dev_bf16(t, name):
     return C.c_void_p(t.data_ptr())
 
 
+class WindowTable:
+    """A window table marshalled once (host int64 array) so that repeated calls pay nothing for it."""
+
+    def __init__(self, table):
+        t = torch.as_tensor(table, dtype=torch.int64).cpu().contiguous()
+        self.n = t.numel()
+        self.arr = (C.c_int64 * self.n)(*t.tolist())
+
+
 def _table_ptr(table, d):
     if table is None:
         return None, None
-    t = torch.as_tensor(table, dtype=torch.int64).cpu().contiguous()
-    if t.numel() != d // 2:
+    wt = table if isinstance(table, WindowTable) else WindowTable(table)
+    if wt.n != d // 2:
         raise AtfError(1, f"table must have d/2 = {d // 2} entries")
-    arr = (C.c_int64 * t.numel())(*t.tolist())
-    return arr, arr
+    return wt.arr, wt
 
 
 _ws = None

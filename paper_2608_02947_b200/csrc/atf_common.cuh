@@ -40,8 +40,8 @@ struct AtfWorkspace {
 };
 AtfWorkspace atf_bound_workspace();
 
-constexpr int ATF_DECODE_TARGET_CTAS = 148 * 4;
-constexpr int ATF_DECODE_MIN_SPLIT = 256;
+constexpr int ATF_DECODE_SLOTS = 148 * 2;  // decode CTAs resident on the GPU at once
+constexpr int ATF_DECODE_MIN_SPLIT = 512;
 int atf_decode_num_splits(int B, int Hkv, int64_t L);
 
 // ------------------------------------------------------------------------------------------

@@ -1,272 +1,371 @@
 // atf_decode: split-K windowed attention of one query row per (batch, head) against a
-// contiguous KV cache (Sec. 5; the last row of Fig. 3).  Bandwidth-bound: every load is a
-// 16-byte vector load, a row of the cache is covered by consecutive lanes, and a lane whose
-// 16-byte chunk of a key row lies wholly outside the key's live pair range issues no load
-// (Sec. 3.3: out-of-window components are not brought on chip).  V rows are read in full.
+// contiguous KV cache (Sec. 5; the last row of Fig. 3).  Bandwidth-bound: the cache is moved
+// with 16-byte asynchronous copies, a row of the cache is covered by consecutive lanes, and a
+// 16-byte chunk of a key row that lies wholly outside the key's live pair range is not read
+// (Sec. 3.3: out-of-window components are not brought on chip) - its place in shared memory is
+// zero-filled instead.  V rows are read in full.
 //
-// Work split: grid = (splits, Hkv, B).  A block owns a contiguous key range; each of its 8
-// warps walks that range in blocks of keys with its own online-softmax state for the G = Hq/Hkv
-// query heads that share the KV head, the warps are merged through shared memory, the block
-// writes one partial (m, l, o) per head, and the last block to finish for a (batch, KV head)
-// merges the partials of all splits by their log-sum-exp and writes O (and LSE).
+// Work split: grid = (splits, Hkv, B).  A block owns a contiguous key range and each of its 4
+// warps walks that range in blocks of 2048/d keys through its own 3-stage cp.async ring.  Per
+// block a warp computes, for the (up to 8) query heads that share the KV head at once:
+//   S = q K^T   with mma.sync (m16n8k16, bf16 in, fp32 accumulate; the heads are the M rows),
+//   the online softmax in registers (log2 domain, lazy rescaling),
+//   O += P V    with mma.sync, V fragments transposed by ldmatrix.
+// The arithmetic is a few instructions per key, so the loads in flight set the speed.  The
+// warps are merged through shared memory, the block writes one partial (m, l, o) per head, and
+// the last block to finish for a (batch, KV head) merges the partials of all splits by their
+// log-sum-exp and writes O (and LSE).
 #include <cfloat>
 
 #include "atf_common.cuh"
 
 namespace {
 
-constexpr int DEC_THREADS = 256;
-constexpr int DEC_WARPS = DEC_THREADS / 32;
-constexpr int DEC_NLD = 8;  // loads in flight per lane for K, and again for V
-
-__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(a), "r"(sel));
-  return d;
-}
+constexpr int DEC_WARPS = 4;
+constexpr int DEC_THREADS = DEC_WARPS * 32;
+constexpr int DEC_STAGES = 3;
+constexpr int DEC_TILE_BYTES = 4096;                               // one K or V block of a warp
+constexpr int DEC_WARP_SMEM = DEC_STAGES * 2 * DEC_TILE_BYTES;     // K and V rings of one warp
+constexpr int DEC_SMEM = DEC_WARPS * DEC_WARP_SMEM;
+constexpr float DEC_RESCALE_THRESHOLD = 8.f;
 
 struct DecodeParams {
   const __nv_bfloat16* q;
   const __nv_bfloat16* K;
   const __nv_bfloat16* V;
   __nv_bfloat16* O;
-  float* lse;            // may be null
-  float* partials;       // [B*Hkv][nsplit][G][D + 2]
-  unsigned int* counters;  // [B*Hkv], zero between launches
+  float* lse;                // may be null
+  float* partials;           // [B*Hkv][nsplit][G][D + 2]
+  unsigned int* counters;    // [B*Hkv], zero between launches
   unsigned long long* kept;  // may be null
-  int Hq, Hkv, L, nsplit, keys_per_split;
+  int Hq, Hkv, G, L, nsplit, keys_per_split;
 };
 
-template <int D, int G, int MODE, bool COUNT>
-__global__ void __launch_bounds__(DEC_THREADS)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, rows 8..15 zero) * B (16x8, bf16)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int D, int MODE, bool COUNT>
+__global__ void __launch_bounds__(DEC_THREADS, 2)
 atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant__ AtfTable table) {
   constexpr int H = D / 2;
-  constexpr int LPR = D / 8;         // lanes per key row (16-byte chunks per row)
-  constexpr int KPL = 32 / LPR;      // keys covered by one warp-wide load
-  constexpr int KB = DEC_NLD * KPL;  // keys per warp iteration
-  constexpr int PSTRIDE = D + 2;     // floats per (split, head) partial: m, l, o[D]
+  constexpr int CPR = D / 8;            // 16-byte chunks per cache row
+  constexpr int ROWB = D * 2;           // bytes per cache row
+  constexpr int KB = DEC_TILE_BYTES / ROWB;  // keys per block (16 for d=128, 32 for d=64)
+  constexpr int NKG = KB / 8;           // groups of 8 keys (MMA N tiles of S)
+  constexpr int NKS = D / 16;           // MMA K steps of q K^T
+  constexpr int NNT = D / 8;            // MMA N tiles of O
+  constexpr int PSTRIDE = D + 2;        // floats per (split, head) partial: m, l, o[D]
+  constexpr int CP_PER_LANE = KB * CPR / 32;
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
+
+  extern __shared__ __align__(128) uint8_t dsm[];
+  __shared__ int sW[ATF_MAX_PAIRS];
+  __shared__ unsigned int s_last;
 
   const int split = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sub = lane / LPR;  // which key of a warp-wide load
-  const int c = lane % LPR;    // 16-byte chunk of the row
-  const int p0 = (c % (LPR / 2)) * 8;  // first pair of the chunk (same in both halves)
-  const int L = P.L;
+  const int g = lane >> 2, t = lane & 3;  // MMA fragment row (query head) and column pair
+  const int G = P.G, L = P.L;
   const int m0 = split * P.keys_per_split;
   const int m1 = min(L, m0 + P.keys_per_split);
   const int64_t slab = ((int64_t)b * P.Hkv + hkv) * (int64_t)L * D;
   const __nv_bfloat16* Kb = P.K + slab;
   const __nv_bfloat16* Vb = P.V + slab;
+  if (threadIdx.x < H) sW[threadIdx.x] = table.w[threadIdx.x];
+  __syncthreads();
+  const int Wmax = sW[H - 1];
 
-  int Wl[8];
+  // A fragments of q for every K step: rows = heads of the group (rows >= G stay zero)
+  uint32_t qa[NKS][2];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) Wl[i] = table.w[p0 + i];
-  const int Wmax = table.w[H - 1];
-
-  // query chunk of each head of the group, pre-multiplied by scale*log2(e)
-  float qf[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const __nv_bfloat16* qp = P.q + ((int64_t)b * P.Hq + hkv * G + g) * D + c * 8;
-    uint4 v = *reinterpret_cast<const uint4*>(qp);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      qf[g][2 * j] = bf16lo_to_f32(w[j]) * kScaleLog2;
-      qf[g][2 * j + 1] = bf16hi_to_f32(w[j]) * kScaleLog2;
+  for (int j = 0; j < NKS; ++j) {
+    qa[j][0] = 0u;
+    qa[j][1] = 0u;
+    if (g < G) {
+      const __nv_bfloat16* qp = P.q + ((int64_t)b * P.Hq + hkv * G + g) * D + 16 * j + 2 * t;
+      qa[j][0] = *reinterpret_cast<const uint32_t*>(qp);
+      qa[j][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
     }
   }
 
-  float mrun[G], lrun[G], o[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    mrun[g] = -INFINITY;
-    lrun[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) o[g][i] = 0.f;
-  }
-  unsigned long long cnt = 0;
+  // this lane's chunk of a cache row in the cp.async mapping, and the widest window among its 8 pairs
+  const int cp_chunk = lane % CPR;
+  const int cp_row0 = lane / CPR;               // first row this lane copies; then every 32/CPR rows
+  const uint32_t warp_smem = smem_u32(dsm) + warp * DEC_WARP_SMEM;
 
-  for (int kb0 = m0 + warp * KB; kb0 < m1; kb0 += DEC_WARPS * KB) {
-    // ---- issue every load of this block of keys ----
-    uint4 kreg[DEC_NLD], vreg[DEC_NLD];
+  auto issue_block = [&](int kb0, int stage) {
+    const uint32_t ks = warp_smem + stage * 2 * DEC_TILE_BYTES, vs = ks + DEC_TILE_BYTES;
 #pragma unroll
-    for (int i = 0; i < DEC_NLD; ++i) {
-      const int key = kb0 + i * KPL + sub;
-      const int z = L - 1 - key;
+    for (int i = 0; i < CP_PER_LANE; ++i) {
+      const int row = cp_row0 + i * (32 / CPR);
+      const int key = kb0 + row;
       const bool valid = key < m1;
-      kreg[i] = make_uint4(0, 0, 0, 0);
-      if (valid && z <= Wl[7]) kreg[i] = ld_nc_v4(Kb + (int64_t)key * D + c * 8);
-    }
-#pragma unroll
-    for (int i = 0; i < DEC_NLD; ++i) {
-      const int key = kb0 + i * KPL + sub;
-      vreg[i] = make_uint4(0, 0, 0, 0);
-      if (key < m1) vreg[i] = ld_nc_v4(Vb + (int64_t)key * D + c * 8);
-    }
-
-    // ---- per-element selectors (exact mode): is the window predicate constant over the block? ----
-    uint32_t sel_lo[4], sel_hi[4];
-    bool uniform = true;
-    if (MODE == ATF_MODE_EXACT) {
-      const int z_near = L - 1 - min(kb0 + KB - 1, m1 - 1);
-      const int z_far = L - 1 - kb0;
-      bool same = true;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) same = same && ((z_near <= Wl[i]) == (z_far <= Wl[i]));
-      uniform = __all_sync(0xffffffffu, same);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        sel_lo[j] = (z_far <= Wl[2 * j]) ? 0x1044u : 0x4444u;
-        sel_hi[j] = (z_far <= Wl[2 * j + 1]) ? 0x3244u : 0x4444u;
-      }
-    }
-
-    // ---- scores ----
-    float s[DEC_NLD][G];
-#pragma unroll
-    for (int i = 0; i < DEC_NLD; ++i) {
-      const int key = kb0 + i * KPL + sub;
+      const int keyc = valid ? key : m1 - 1;
       const int z = L - 1 - key;
-      const uint32_t w[4] = {kreg[i].x, kreg[i].y, kreg[i].z, kreg[i].w};
-      float kf[8];
-      if (MODE == ATF_MODE_EXACT) {
-        if (!uniform) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            sel_lo[j] = (z <= Wl[2 * j]) ? 0x1044u : 0x4444u;
-            sel_hi[j] = (z <= Wl[2 * j + 1]) ? 0x3244u : 0x4444u;
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          kf[2 * j] = __uint_as_float(prmt(w[j], sel_lo[j]));
-          kf[2 * j + 1] = __uint_as_float(prmt(w[j], sel_hi[j]));
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          kf[2 * j] = bf16lo_to_f32(w[j]);
-          kf[2 * j + 1] = bf16hi_to_f32(w[j]);
-        }
-      }
-      if (COUNT) {
-        if (key < m1 && c < LPR / 2) {
-          if (MODE == ATF_MODE_EXACT) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) cnt += (z <= Wl[e]) ? 1 : 0;
-          } else {
-            cnt += (z <= Wl[7]) ? 8 : 0;
-          }
-        }
-      }
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float a = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a = fmaf(qf[g][e], kf[e], a);
-#pragma unroll
-        for (int off = 1; off < LPR; off <<= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-        s[i][g] = (key < m1 && z <= Wmax) ? a : -INFINITY;
-      }
+      const uint32_t off = row * ROWB + ((cp_chunk ^ (row & 7)) << 4);
+      const int64_t goff = (int64_t)keyc * D + cp_chunk * 8;
+      // A 128-byte half row always ends in live low-frequency pairs, and DRAM moves whole
+      // 128-byte lines, so leaving out the dead 16-byte chunks of a row would save no traffic:
+      // rows are copied whole (a key no pair reaches is not copied at all) and the dead
+      // elements are masked in registers.
+      cp_async16(ks + off, Kb + goff, (valid && z <= Wmax) ? 16 : 0);
+      cp_async16(vs + off, Vb + goff, (valid && z <= Wmax) ? 16 : 0);
     }
+  };
 
-    // ---- online softmax (log2 domain) and P*V ----
+  float oacc[NNT][4];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float bm = s[0][g];
+  for (int nt = 0; nt < NNT; ++nt)
 #pragma unroll
-      for (int i = 1; i < DEC_NLD; ++i) bm = fmaxf(bm, s[i][g]);
-#pragma unroll
-      for (int off = LPR; off < 32; off <<= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, off));
-      const float mnew = fmaxf(mrun[g], bm);
-      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
-      const float alpha = exp2f(mrun[g] - msafe);
-      mrun[g] = mnew;
-      float psum = 0.f;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[g][e] *= alpha;
-#pragma unroll
-      for (int i = 0; i < DEC_NLD; ++i) {
-        const float p = exp2f(s[i][g] - msafe);
-        psum += p;
-        const uint32_t w[4] = {vreg[i].x, vreg[i].y, vreg[i].z, vreg[i].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          o[g][2 * j] = fmaf(p, bf16lo_to_f32(w[j]), o[g][2 * j]);
-          o[g][2 * j + 1] = fmaf(p, bf16hi_to_f32(w[j]), o[g][2 * j + 1]);
-        }
-      }
-      lrun[g] = lrun[g] * alpha + psum;
-    }
+    for (int e = 0; e < 4; ++e) oacc[nt][e] = 0.f;
+  float m_used = -INFINITY, l_part = 0.f;  // row g of this lane; l_part over this lane's key columns
+  unsigned long long cnt = 0;
+  int r_far = 0;  // first live pair at the far end of the current block (cursor: only moves down as keys advance)
+  {
+    const int z0 = L - 1 - (m0 + warp * KB);
+    while (r_far < H && sW[r_far] < z0) ++r_far;
   }
 
-  // ---- merge the key sub-groups of the warp (they share mrun) ----
+  // ---- prologue: fill the ring ----
+  const int kb_first = m0 + warp * KB;
+  const int kb_step = DEC_WARPS * KB;
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-#pragma unroll
-    for (int off = LPR; off < 32; off <<= 1) {
-      lrun[g] += __shfl_xor_sync(0xffffffffu, lrun[g], off);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) o[g][e] += __shfl_xor_sync(0xffffffffu, o[g][e], off);
-    }
+  for (int s = 0; s < DEC_STAGES - 1; ++s) {
+    const int kb0 = kb_first + s * kb_step;
+    if (kb0 < m1) issue_block(kb0, s);
+    cp_async_commit();
   }
 
-  // ---- merge the warps of the block ----
-  extern __shared__ float sm[];  // [DEC_WARPS][G][PSTRIDE]
-  if (sub == 0) {
+  int it = 0;
+  for (int kb0 = kb_first; kb0 < m1; kb0 += kb_step, ++it) {
+    cp_async_wait<DEC_STAGES - 2>();
+    __syncwarp();
+    {
+      const int kbn = kb0 + (DEC_STAGES - 1) * kb_step;
+      if (kbn < m1) issue_block(kbn, (it + DEC_STAGES - 1) % DEC_STAGES);
+      cp_async_commit();
+    }
+    const uint32_t ks = warp_smem + (it % DEC_STAGES) * 2 * DEC_TILE_BYTES, vs = ks + DEC_TILE_BYTES;
+
+    // ---- live pair range over the block (coarse mode: first live pair rounded down to 8) ----
+    const int z_far = L - 1 - kb0;                      // the block's first key is the farthest
+    const int z_near = max(L - 1 - (kb0 + KB - 1), 0);
+    while (r_far > 0 && sW[r_far - 1] >= z_far) --r_far;
+    int r_near = r_far;
+    while (r_near > 0 && sW[r_near - 1] >= z_near) --r_near;
+    const int rq_far = MODE == ATF_MODE_COARSE ? (r_far >= H ? H : (r_far & ~7)) : r_far;
+    const int rq_near = MODE == ATF_MODE_COARSE ? (r_near & ~7) : r_near;
+    const bool uniform = rq_near == rq_far;
+    // K steps (16 pairs of one half) below the nearest key's first live pair are dead for every key
+    const int jl = rq_near >> 4;
+    // element masks of the K step that holds a first live pair r: lane t holds pairs 2t, 2t+1 of the
+    // step's first chunk and 8+2t, 9+2t of its second chunk
+    auto step_masks = [&](int r, uint32_t& mk0, uint32_t& mk1) {
+      const int e = r & 15;
+      mk0 = ((2 * t >= e) ? 0x0000FFFFu : 0u) | ((2 * t + 1 >= e) ? 0xFFFF0000u : 0u);
+      mk1 = ((8 + 2 * t >= e) ? 0x0000FFFFu : 0u) | ((9 + 2 * t >= e) ? 0xFFFF0000u : 0u);
+    };
+    uint32_t mku0 = 0xFFFFFFFFu, mku1 = 0xFFFFFFFFu;
+    if (uniform) step_masks(rq_far, mku0, mku1);
+    // general blocks (the block straddles a window boundary): first live pair of this lane's key in each group
+    int r_lane[NKG];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float* dst = sm + ((warp * G + g) * PSTRIDE);
-      if (c == 0) {
-        dst[0] = mrun[g];
-        dst[1] = lrun[g];
+    for (int kg = 0; kg < NKG; ++kg) r_lane[kg] = rq_far;
+    if (!uniform) {
+#pragma unroll
+      for (int kg = 0; kg < NKG; ++kg) {
+        const int z = L - 1 - (kb0 + kg * 8 + g);
+        int r = r_near;
+        while (r < r_far && sW[r] < z) ++r;
+        r_lane[kg] = MODE == ATF_MODE_COARSE ? (r >= H ? H : (r & ~7)) : r;
       }
+    }
+
+    // ---- S = q K^T ----
+    float sc[NKG][4];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) dst[2 + c * 8 + e] = o[g][e];
+    for (int kg = 0; kg < NKG; ++kg)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) sc[kg][e] = 0.f;
+#pragma unroll
+    for (int j = 0; j < NKS; ++j) {
+      const int jh = j % (NKS / 2);  // K step within its half
+      if (jh < jl) continue;         // warp-uniform
+#pragma unroll
+      for (int kp = 0; kp < NKG / 2; ++kp) {
+        // matrices: (group 2kp, chunk 2j), (group 2kp, chunk 2j+1), (group 2kp+1, chunk 2j), (group 2kp+1, chunk 2j+1)
+        const int mi = lane >> 3, mr = lane & 7;
+        const int row = (2 * kp + (mi >> 1)) * 8 + mr;
+        const int chunk = 2 * j + (mi & 1);
+        uint32_t bf[4];
+        ldsm_x4(ks + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
+        if (uniform) {
+          if (jh == (rq_far >> 4)) {
+            bf[0] &= mku0;
+            bf[1] &= mku1;
+            bf[2] &= mku0;
+            bf[3] &= mku1;
+          }
+        } else {
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int r = r_lane[2 * kp + h2];
+            uint32_t mk0 = 0xFFFFFFFFu, mk1 = 0xFFFFFFFFu;
+            if (jh < (r >> 4)) {
+              mk0 = 0u;
+              mk1 = 0u;
+            } else if (jh == (r >> 4)) {
+              step_masks(r, mk0, mk1);
+            }
+            bf[2 * h2] &= mk0;
+            bf[2 * h2 + 1] &= mk1;
+          }
+        }
+        mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
+        mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
+      }
+    }
+    if (COUNT) {
+      // one lane per key: lanes t == 0 own key (group, g)
+      if (t == 0) {
+#pragma unroll
+        for (int kg = 0; kg < NKG; ++kg) {
+          const int key = kb0 + kg * 8 + g;
+          if (key < m1) cnt += (unsigned long long)(H - r_lane[kg]);
+        }
+      }
+    }
+
+    // ---- online softmax (log2 domain); this lane holds keys 2t, 2t+1 of every group for head g ----
+    float mx = -INFINITY;
+#pragma unroll
+    for (int kg = 0; kg < NKG; ++kg) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int key = kb0 + kg * 8 + 2 * t + e;
+        const int z = L - 1 - key;
+        sc[kg][e] = (key < m1 && z <= Wmax) ? sc[kg][e] * kScaleLog2 : -INFINITY;
+        mx = fmaxf(mx, sc[kg][e]);
+      }
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    float scale_o = 1.f;
+    bool moved = false;
+    if (mx > m_used + (m_used == -INFINITY ? 0.f : DEC_RESCALE_THRESHOLD)) {
+      scale_o = (m_used == -INFINITY) ? 0.f : ex2f(m_used - mx);
+      m_used = mx;
+      moved = true;
+    }
+    if (__any_sync(0xffffffffu, moved)) {
+      l_part *= scale_o;
+#pragma unroll
+      for (int nt = 0; nt < NNT; ++nt) {
+        oacc[nt][0] *= scale_o;
+        oacc[nt][1] *= scale_o;
+      }
+    }
+    const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+    uint32_t pa[NKG];
+#pragma unroll
+    for (int kg = 0; kg < NKG; ++kg) {
+      const float p0 = ex2f(sc[kg][0] - mref), p1 = ex2f(sc[kg][1] - mref);
+      l_part += p0 + p1;
+      pa[kg] = pack_bf16x2(p0, p1);
+    }
+
+    // ---- O += P V ----
+#pragma unroll
+    for (int pk = 0; pk < NKG / 2; ++pk) {
+#pragma unroll
+      for (int np = 0; np < NNT / 2; ++np) {
+        // matrices: (keys 0-7, chunk 2np), (keys 8-15, chunk 2np), (keys 0-7, chunk 2np+1), (keys 8-15, chunk 2np+1)
+        const int mi = lane >> 3, mr = lane & 7;
+        const int row = pk * 16 + (mi & 1) * 8 + mr;
+        const int chunk = 2 * np + (mi >> 1);
+        uint32_t bf[4];
+        ldsm_x4_trans(vs + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
+        mma_bf16_16816(oacc[2 * np], pa[2 * pk], pa[2 * pk + 1], bf[0], bf[1]);
+        mma_bf16_16816(oacc[2 * np + 1], pa[2 * pk], pa[2 * pk + 1], bf[2], bf[3]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+  // ---- merge the warps of the block (the rings are free now) ----
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+  __syncthreads();
+  float* sm = reinterpret_cast<float*>(dsm);  // [DEC_WARPS][G][PSTRIDE]
+  if (g < G) {
+    float* dst = sm + (warp * G + g) * PSTRIDE;
+    if (t == 0) {
+      dst[0] = m_used;
+      dst[1] = l_part;
+    }
+#pragma unroll
+    for (int nt = 0; nt < NNT; ++nt) {
+      dst[2 + nt * 8 + 2 * t] = oacc[nt][0];
+      dst[2 + nt * 8 + 2 * t + 1] = oacc[nt][1];
     }
   }
   __syncthreads();
   const int64_t grp = (int64_t)b * P.Hkv + hkv;
   float* part = P.partials + (grp * P.nsplit + split) * (int64_t)(G * PSTRIDE);
   for (int idx = threadIdx.x; idx < G * D; idx += DEC_THREADS) {
-    const int g = idx / D, col = idx % D;
+    const int gg = idx / D, col = idx % D;
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm[(w * G + g) * PSTRIDE]);
+    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm[(w * G + gg) * PSTRIDE]);
     const float Ms = (M == -INFINITY) ? 0.f : M;
     float acc = 0.f, lacc = 0.f;
 #pragma unroll
     for (int w = 0; w < DEC_WARPS; ++w) {
-      const float* src = sm + (w * G + g) * PSTRIDE;
-      const float f = exp2f(src[0] - Ms);
+      const float* src = sm + (w * G + gg) * PSTRIDE;
+      const float f = ex2f(src[0] - Ms);
       acc += f * src[2 + col];
       lacc += f * src[1];
     }
-    part[g * PSTRIDE + 2 + col] = acc;
+    part[gg * PSTRIDE + 2 + col] = acc;
     if (col == 0) {
-      part[g * PSTRIDE] = M;
-      part[g * PSTRIDE + 1] = lacc;
+      part[gg * PSTRIDE] = M;
+      part[gg * PSTRIDE + 1] = lacc;
     }
   }
   if (COUNT) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
     if (lane == 0 && cnt) {
-      for (int g = 0; g < G; ++g) atomicAdd(P.kept + (int64_t)b * P.Hq + hkv * G + g, cnt);
+      for (int gg = 0; gg < G; ++gg) atomicAdd(P.kept + (int64_t)b * P.Hq + hkv * G + gg, cnt);
     }
   }
 
   // ---- last block of this (batch, KV head) merges all splits ----
-  __shared__ unsigned int s_last;
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -278,46 +377,45 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   __threadfence();
   const float* allp = P.partials + grp * P.nsplit * (int64_t)(G * PSTRIDE);
   // one warp per head: lanes stride over the splits for the LSE merge, then over columns
-  for (int g = warp; g < G; g += DEC_WARPS) {
+  for (int gg = warp; gg < G; gg += DEC_WARPS) {
     float M = -INFINITY;
-    for (int sp = lane; sp < P.nsplit; sp += 32) M = fmaxf(M, __ldcg(allp + ((int64_t)sp * G + g) * PSTRIDE));
+    for (int sp = lane; sp < P.nsplit; sp += 32) M = fmaxf(M, __ldcg(allp + ((int64_t)sp * G + gg) * PSTRIDE));
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
     const float Ms = (M == -INFINITY) ? 0.f : M;
     float Lsum = 0.f;
     for (int sp = lane; sp < P.nsplit; sp += 32) {
-      const float* src = allp + ((int64_t)sp * G + g) * PSTRIDE;
-      Lsum += exp2f(__ldcg(src) - Ms) * __ldcg(src + 1);
+      const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
+      Lsum += ex2f(__ldcg(src) - Ms) * __ldcg(src + 1);
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, off);
     const float inv = 1.f / Lsum;
     float acc[D / 32];
 #pragma unroll
-    for (int t = 0; t < D / 32; ++t) acc[t] = 0.f;
+    for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
     for (int sp = 0; sp < P.nsplit; ++sp) {
-      const float* src = allp + ((int64_t)sp * G + g) * PSTRIDE;
-      const float f = exp2f(__ldcg(src) - Ms);
+      const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
+      const float f = ex2f(__ldcg(src) - Ms);
 #pragma unroll
-      for (int t = 0; t < D / 32; ++t) acc[t] = fmaf(f, __ldcg(src + 2 + t * 32 + lane), acc[t]);
+      for (int c = 0; c < D / 32; ++c) acc[c] = fmaf(f, __ldcg(src + 2 + c * 32 + lane), acc[c]);
     }
-    const int64_t hq = (int64_t)b * P.Hq + hkv * G + g;
+    const int64_t hq = (int64_t)b * P.Hq + hkv * G + gg;
 #pragma unroll
-    for (int t = 0; t < D / 32; ++t) P.O[hq * D + t * 32 + lane] = __float2bfloat16_rn(acc[t] * inv);
+    for (int c = 0; c < D / 32; ++c) P.O[hq * D + c * 32 + lane] = __float2bfloat16_rn(acc[c] * inv);
     if (P.lse && lane == 0) P.lse[hq] = (Ms + log2f(Lsum)) * 0.6931471805599453f;
   }
   if (threadIdx.x == 0) P.counters[grp] = 0;  // ready for the next launch
 }
 
-template <int D, int G>
+template <int D>
 atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
   dim3 grid(P.nsplit, P.Hkv, B);
-  const size_t smem = (size_t)DEC_WARPS * G * (D + 2) * sizeof(float);
 #define ATF_DEC_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                  \
-    auto kern = atf_decode_kernel<D, G, MODE_, COUNT_>;                                                 \
-    if (smem > 48 * 1024) ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    kern<<<grid, DEC_THREADS, smem, s>>>(P, t);                                                         \
+    auto kern = atf_decode_kernel<D, MODE_, COUNT_>;                                                    \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DEC_SMEM));  \
+    kern<<<grid, DEC_THREADS, DEC_SMEM, s>>>(P, t);                                                     \
   } while (0)
   if (mode == ATF_MODE_EXACT) {
     if (count) ATF_DEC_LAUNCH(ATF_MODE_EXACT, true); else ATF_DEC_LAUNCH(ATF_MODE_EXACT, false);
@@ -327,21 +425,6 @@ atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mo
 #undef ATF_DEC_LAUNCH
   ATF_CUDA_CHECK(cudaGetLastError());
   return ATF_OK;
-}
-
-template <int D>
-atf_status dispatch_group(int G, const DecodeParams& P, const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
-  switch (G) {
-    case 1: return launch_decode<D, 1>(P, t, B, mode, count, s);
-    case 2: return launch_decode<D, 2>(P, t, B, mode, count, s);
-    case 3: return launch_decode<D, 3>(P, t, B, mode, count, s);
-    case 4: return launch_decode<D, 4>(P, t, B, mode, count, s);
-    case 5: return launch_decode<D, 5>(P, t, B, mode, count, s);
-    case 6: return launch_decode<D, 6>(P, t, B, mode, count, s);
-    case 7: return launch_decode<D, 7>(P, t, B, mode, count, s);
-    case 8: return launch_decode<D, 8>(P, t, B, mode, count, s);
-    default: return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: Hq/Hkv must be in 1..8 (got %d)", G);
-  }
 }
 
 }  // namespace
@@ -363,6 +446,7 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: d must be 64 or 128 (got %d)", d);
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: bad shape");
   if (Hq % Hkv) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: Hq must be a multiple of Hkv");
+  if (Hq / Hkv > 8) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: Hq/Hkv must be at most 8 (got %d)", Hq / Hkv);
   if (L * (int64_t)d >= (1ll << 31)) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: L*d must be below 2^31");
   if (B > 65535 || Hkv > 65535 || (int64_t)B * Hkv > ATF_WS_COUNTER_SLOTS)
     return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: B*Hkv must be <= %d", ATF_WS_COUNTER_SLOTS);
@@ -390,9 +474,10 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.kept = opts ? (unsigned long long*)opts->kept_terms : nullptr;
   P.Hq = Hq;
   P.Hkv = Hkv;
+  P.G = Hq / Hkv;
   P.L = (int)L;
   P.nsplit = atf_decode_num_splits(B, Hkv, L);
-  const int kb = 8 * (32 / (d / 8));  // keys per warp iteration
+  const int kb = 2048 / d;  // keys per warp iteration
   int64_t kps = (L + P.nsplit - 1) / P.nsplit;
   kps = (kps + kb - 1) / kb * kb;
   P.keys_per_split = (int)kps;
@@ -402,8 +487,7 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.partials = (float*)(base + ATF_WS_HEADER);
   cudaStream_t s = (cudaStream_t)stream;
   const bool count = P.kept != nullptr;
-  return d == 64 ? dispatch_group<64>(Hq / Hkv, P, t, B, mode, count, s)
-                 : dispatch_group<128>(Hq / Hkv, P, t, B, mode, count, s);
+  return d == 64 ? launch_decode<64>(P, t, B, mode, count, s) : launch_decode<128>(P, t, B, mode, count, s);
 }
 
 extern "C" atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, void* O, int B, int Hq,

@@ -20,13 +20,27 @@ atf_status atf_fail(atf_status code, const char* fmt, ...) {
 
 AtfWorkspace atf_bound_workspace() { return g_ws; }
 
+// Splits of the key range per (batch, KV head) for decode.  Two decode CTAs fit on each of
+// the 148 SMs; pick the smallest split count that fills whole waves of those 296 slots best,
+// with at least ATF_DECODE_MIN_SPLIT keys per split.
 int atf_decode_num_splits(int B, int Hkv, int64_t L) {
-  int64_t groups = (int64_t)B * Hkv;
-  int64_t want = (ATF_DECODE_TARGET_CTAS + groups - 1) / groups;
-  int64_t most = (L + ATF_DECODE_MIN_SPLIT - 1) / ATF_DECODE_MIN_SPLIT;
-  if (want > most) want = most;
-  if (want < 1) want = 1;
-  return (int)want;
+  const int64_t groups = (int64_t)B * Hkv;
+  const int64_t slots = ATF_DECODE_SLOTS;
+  int64_t most = L / ATF_DECODE_MIN_SPLIT;
+  if (most < 1) most = 1;
+  if (most > 4 * slots) most = 4 * slots;
+  double best = -1.0;
+  int best_ns = 1;
+  for (int64_t ns = 1; ns <= most; ++ns) {
+    const int64_t total = groups * ns;
+    const int64_t waves = (total + slots - 1) / slots;
+    const double eff = (double)total / (double)(waves * slots);
+    if (eff > best + 0.02) {
+      best = eff;
+      best_ns = (int)ns;
+    }
+  }
+  return best_ns;
 }
 
 // Checks a caller's table (host, d/2 entries; NULL = full attention) and converts it to the

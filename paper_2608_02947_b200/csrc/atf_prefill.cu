@@ -132,7 +132,7 @@ __device__ __forceinline__ int tile_depth(int H, int p_any, int p_mid, int dt) {
 // of 2^f on f = x - n in [-0.5, 0.5] (relative error < 8e-5, below the bf16 rounding of P),
 // and add n to the exponent field.
 #ifndef ATF_POLY_OF_4
-#define ATF_POLY_OF_4 2
+#define ATF_POLY_OF_4 0
 #endif
 constexpr int POLY_OF_4 = ATF_POLY_OF_4;  // of every 4 packed pairs, this many take the polynomial, the rest MUFU
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
