@@ -61,6 +61,18 @@ typedef struct {
   int64_t original_ctx;
 } atf_scaling;
 
+/* Layout of the K cache handed to atf_decode_ex.
+ * ATF_KLAYOUT_ROWS  : [B, Hkv, L, d], the layout of K in atf_prefill (default).
+ * ATF_KLAYOUT_GROUPS: [B, Hkv, T, d/16, KT, 16] as written by atf_kcache_pack: the keys are cut
+ *   into T = ceil(L/KT) tiles of KT = atf_kcache_tile_keys(d) keys (16 KiB per tile); inside a
+ *   tile, group j holds, for each of its keys, the 8 pairs r = d/2-1-8j ... d/2-8-8j (lowest
+ *   frequency first), each pair as (dim r, dim r + d/2) side by side.  The pairs a far key
+ *   keeps (a low-frequency slice, Sec. 3.3) are then the leading groups, i.e. a contiguous
+ *   prefix of the tile, so decode fetches only live bytes; in the row layout DRAM's 128-byte
+ *   lines make it fetch every row whole.  This layout is an extension: the paper's ports keep
+ *   the row layout.                                                                          */
+enum { ATF_KLAYOUT_ROWS = 0, ATF_KLAYOUT_GROUPS = 1 };
+
 /* Optional arguments of the *_ex calls.  Zero-initialise, then set what is needed. */
 typedef struct {
   int mode;              /* ATF_MODE_EXACT or ATF_MODE_COARSE                                  */
@@ -70,6 +82,7 @@ typedef struct {
   float* lse;            /* decode only: dev, [B*Hq] fp32 natural-log LSE, or NULL              */
   void* workspace;       /* dev scratch for this call, or NULL to use the bound workspace       */
   size_t workspace_bytes;
+  int k_layout;          /* decode only: ATF_KLAYOUT_ROWS (default) or ATF_KLAYOUT_GROUPS        */
 } atf_opts;
 
 /* Window table (Eq. 2, Eq. 3; effective frequencies per Sec. 3.2).  Host only, no GPU needed.
@@ -117,6 +130,16 @@ atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, voi
 atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, void* O, int B,
                          int Hq, int Hkv, int64_t L, int d, const int64_t* table,
                          const atf_opts* opts, void* stream);
+
+/* Copies n rotated key rows into a group-major K cache (see ATF_KLAYOUT_GROUPS; Sec. 3.3's
+ * "out-of-window components are not loaded" made to hold at DRAM line granularity).
+ *   K : dev bf16 [B, Hkv, n, d], rows for positions pos0 .. pos0+n-1;
+ *   Kg: dev bf16 [B, Hkv, ceil(Lcap/KT), d/16, KT, 16], the cache, Lcap >= pos0 + n its length
+ *       in keys, KT = atf_kcache_tile_keys(d) (64 for d = 128, 128 for d = 64).
+ * atf_decode_ex with k_layout = ATF_KLAYOUT_GROUPS then wants ceil(L/KT) == ceil(Lcap/KT).    */
+int64_t atf_kcache_tile_keys(int d);
+atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, int64_t n, int64_t Lcap,
+                           int64_t pos0, int d, void* stream);
 
 /* Workspace.  The library keeps no allocation of its own: the caller allocates
  * atf_workspace_bytes() bytes of device memory (256-byte aligned), zero-fills it once, and

@@ -10,6 +10,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 ATF_MODE_EXACT, ATF_MODE_COARSE = 0, 1
 ATF_OP_PREFILL, ATF_OP_DECODE = 0, 1
+ATF_KLAYOUT_ROWS, ATF_KLAYOUT_GROUPS = 0, 1
 
 
 class AtfError(RuntimeError):
@@ -25,7 +26,7 @@ class _Scaling(C.Structure):
 
 class _Opts(C.Structure):
     _fields_ = [("mode", C.c_int), ("kept_terms", C.c_void_p), ("lse", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("k_layout", C.c_int)]
 
 
 def lib_path():
@@ -53,12 +54,16 @@ def lib():
     L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
     L.atf_decode.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
     L.atf_decode_ex.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), C.POINTER(_Opts), vp]
+    L.atf_kcache_pack.argtypes = [vp, vp, i, i, i64, i64, i64, i, vp]
+    L.atf_kcache_tile_keys.argtypes = [i]
+    L.atf_kcache_tile_keys.restype = C.c_int64
     L.atf_workspace_bytes.argtypes = [i, i, i, i, i64, i]
     L.atf_workspace_bytes.restype = C.c_size_t
     L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
     L.atf_check_status.argtypes = [vp]
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_decode", "atf_decode_ex",
+                 "atf_kcache_pack",
                  "atf_bind_workspace", "atf_check_status"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -144,11 +149,12 @@ def atf_rope(X, theta, pos0=0):
     return X
 
 
-def _opts(mode, kept_terms, lse):
-    if mode == ATF_MODE_EXACT and kept_terms is None and lse is None:
+def _opts(mode, kept_terms, lse, k_layout=ATF_KLAYOUT_ROWS):
+    if mode == ATF_MODE_EXACT and kept_terms is None and lse is None and k_layout == ATF_KLAYOUT_ROWS:
         return None
     o = _Opts()
     o.mode = int(mode)
+    o.k_layout = int(k_layout)
     o.kept_terms = kept_terms.data_ptr() if kept_terms is not None else None
     o.lse = lse.data_ptr() if lse is not None else None
     o.workspace = None
@@ -193,23 +199,47 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
     return O, LSE
 
 
+def atf_kcache_pack(K, Kg=None, pos0=0):
+    """Copies rotated key rows K [B,Hkv,n,d] into a tiled group-major cache
+    Kg [B,Hkv,tiles,d/16,KT,16] at positions pos0.. (allocates a zeroed cache for exactly pos0+n keys
+    if Kg is None). Returns Kg."""
+    _dev_bf16(K, "K")
+    B, Hkv, n, d = K.shape
+    kt = int(lib().atf_kcache_tile_keys(d))
+    if Kg is None:
+        Kg = torch.zeros((B, Hkv, (pos0 + n + kt - 1) // kt, d // 16, kt, 16), dtype=torch.bfloat16, device=K.device)
+    _dev_bf16(Kg, "Kg")
+    if Kg.dim() != 6 or Kg.shape[:2] != (B, Hkv) or Kg.shape[3:] != (d // 16, kt, 16):
+        raise AtfError(1, f"Kg must be [B,Hkv,tiles,d/16,{kt},16]")
+    _check(lib().atf_kcache_pack(C.c_void_p(K.data_ptr()), C.c_void_p(Kg.data_ptr()), B, Hkv, n, Kg.shape[2] * kt,
+                                 int(pos0), d, _stream(K)))
+    return Kg
+
+
 def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=False, O=None):
-    """One decode step: q [B,Hq,d] at position L-1 against Kcache/Vcache [B,Hkv,L,d] (bf16)."""
+    """One decode step: q [B,Hq,d] at position L-1 against Kcache/Vcache [B,Hkv,L,d] (bf16).
+    Kcache may also be a tiled group-major cache [B,Hkv,tiles,d/16,KT,16] from atf_kcache_pack."""
     on_host = not q.is_cuda
     if on_host:
         q, Kcache, Vcache = _host_roundtrip([q, Kcache, Vcache])
     for t, nm in ((q, "q"), (Kcache, "Kcache"), (Vcache, "Vcache")):
         _dev_bf16(t, nm)
     B, Hq, d = q.shape
-    Hkv, L = Kcache.shape[1], Kcache.shape[2]
-    if Kcache.shape != (B, Hkv, L, d) or Vcache.shape != Kcache.shape:
-        raise AtfError(1, "Kcache and Vcache must be [B,Hkv,L,d] matching q")
+    Hkv, L = Vcache.shape[1], Vcache.shape[2]
+    k_layout = ATF_KLAYOUT_GROUPS if Kcache.dim() == 6 else ATF_KLAYOUT_ROWS
+    if k_layout == ATF_KLAYOUT_GROUPS:
+        kt = int(lib().atf_kcache_tile_keys(d))
+        want_k = (B, Hkv, (L + kt - 1) // kt, d // 16, kt, 16)
+    else:
+        want_k = (B, Hkv, L, d)
+    if Vcache.shape != (B, Hkv, L, d) or tuple(Kcache.shape) != want_k:
+        raise AtfError(1, "Vcache must be [B,Hkv,L,d] and Kcache [B,Hkv,L,d] or [B,Hkv,tiles,d/16,KT,16], matching q")
     if O is None:
         O = torch.empty_like(q)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
     ensure_workspace(atf_workspace_bytes(ATF_OP_DECODE, B, Hq, Hkv, L, d), q.device)
     tab, _keep = _table_ptr(table, d)
-    o = _opts(mode, kept_terms, lse)
+    o = _opts(mode, kept_terms, lse, k_layout)
     _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
                                C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,
                                C.byref(o) if o is not None else None, _stream(q)))

@@ -69,7 +69,7 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-template <int D, int MODE, bool COUNT>
+template <int D, int MODE, bool COUNT, int KL>
 __global__ void __launch_bounds__(DEC_THREADS, 2)
 atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant__ AtfTable table) {
   constexpr int H = D / 2;
@@ -81,6 +81,7 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   constexpr int NNT = D / 8;            // MMA N tiles of O
   constexpr int PSTRIDE = D + 2;        // floats per (split, head) partial: m, l, o[D]
   constexpr int CP_PER_LANE = KB * CPR / 32;
+  constexpr int KT = DEC_WARPS * KB;    // keys per tile of the group-major K cache (one block per warp)
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
 
   extern __shared__ __align__(128) uint8_t dsm[];
@@ -94,22 +95,34 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   const int m0 = split * P.keys_per_split;
   const int m1 = min(L, m0 + P.keys_per_split);
   const int64_t slab = ((int64_t)b * P.Hkv + hkv) * (int64_t)L * D;
-  const __nv_bfloat16* Kb = P.K + slab;
-  const __nv_bfloat16* Vb = P.V + slab;
+  // the group-major cache is padded to whole tiles of DEC_WARPS * KB keys
+  const __nv_bfloat16* Kb = P.K + (KL == ATF_KLAYOUT_ROWS
+                                       ? slab
+                                       : ((int64_t)b * P.Hkv + hkv) * (((int64_t)L + DEC_WARPS * KB - 1) / (DEC_WARPS * KB)) *
+                                             (int64_t)(DEC_WARPS * KB) * D);
   if (threadIdx.x < H) sW[threadIdx.x] = table.w[threadIdx.x];
   __syncthreads();
   const int Wmax = sW[H - 1];
 
-  // A fragments of q for every K step: rows = heads of the group (rows >= G stay zero)
+  // A fragments of q for every K step: rows = heads of the group (rows >= G stay zero).
+  // Row layout: K step j contracts dims 16j..16j+15.  Group-major layout: K step j contracts the
+  // 8 pairs of group j, lowest frequency first, each pair as (dim r, dim r + h) side by side.
   uint32_t qa[NKS][2];
 #pragma unroll
   for (int j = 0; j < NKS; ++j) {
     qa[j][0] = 0u;
     qa[j][1] = 0u;
     if (g < G) {
-      const __nv_bfloat16* qp = P.q + ((int64_t)b * P.Hq + hkv * G + g) * D + 16 * j + 2 * t;
-      qa[j][0] = *reinterpret_cast<const uint32_t*>(qp);
-      qa[j][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
+      const __nv_bfloat16* qrow = P.q + ((int64_t)b * P.Hq + hkv * G + g) * D;
+      if (KL == ATF_KLAYOUT_ROWS) {
+        qa[j][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t);
+        qa[j][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 8 + 2 * t);
+      } else {
+        const int ra = H - 1 - (8 * j + t), rb = H - 1 - (8 * j + 4 + t);
+        const uint16_t* q16 = reinterpret_cast<const uint16_t*>(qrow);
+        qa[j][0] = (uint32_t)q16[ra] | ((uint32_t)q16[ra + H] << 16);
+        qa[j][1] = (uint32_t)q16[rb] | ((uint32_t)q16[rb + H] << 16);
+      }
     }
   }
 
@@ -118,23 +131,50 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   const int cp_row0 = lane / CPR;               // first row this lane copies; then every 32/CPR rows
   const uint32_t warp_smem = smem_u32(dsm) + warp * DEC_WARP_SMEM;
 
+  const __nv_bfloat16* Vb = P.V + slab;
+  int r_iss = 0;  // cursor for the copies: first live pair of the nearest key of the block being fetched
   auto issue_block = [&](int kb0, int stage) {
     const uint32_t ks = warp_smem + stage * 2 * DEC_TILE_BYTES, vs = ks + DEC_TILE_BYTES;
+    // V rows, and K rows in the row layout, are copied whole: a 128-byte half row always ends in
+    // live low-frequency pairs and DRAM moves whole 128-byte lines, so leaving out dead 16-byte
+    // chunks of a row would save no traffic.  A key no pair reaches is not copied at all.
 #pragma unroll
     for (int i = 0; i < CP_PER_LANE; ++i) {
       const int row = cp_row0 + i * (32 / CPR);
       const int key = kb0 + row;
-      const bool valid = key < m1;
-      const int keyc = valid ? key : m1 - 1;
-      const int z = L - 1 - key;
+      const bool valid = key < m1 && (L - 1 - key) <= Wmax;
+      const int keyc = key < m1 ? key : m1 - 1;
       const uint32_t off = row * ROWB + ((cp_chunk ^ (row & 7)) << 4);
       const int64_t goff = (int64_t)keyc * D + cp_chunk * 8;
-      // A 128-byte half row always ends in live low-frequency pairs, and DRAM moves whole
-      // 128-byte lines, so leaving out the dead 16-byte chunks of a row would save no traffic:
-      // rows are copied whole (a key no pair reaches is not copied at all) and the dead
-      // elements are masked in registers.
-      cp_async16(ks + off, Kb + goff, (valid && z <= Wmax) ? 16 : 0);
-      cp_async16(vs + off, Vb + goff, (valid && z <= Wmax) ? 16 : 0);
+      if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + off, Kb + goff, valid ? 16 : 0);
+      cp_async16(vs + off, Vb + goff, valid ? 16 : 0);
+    }
+    if (KL == ATF_KLAYOUT_GROUPS) {
+      // group-major K: the live pairs of a key are its first groups, each group a contiguous
+      // stream over the keys, so only live bytes are fetched (8-pair granularity)
+      const int z_near = max(L - 1 - (kb0 + KB - 1), 0);
+      if (r_iss >= H || sW[r_iss] < z_near) {
+        r_iss = 0;
+        while (r_iss < H && sW[r_iss] < z_near) ++r_iss;
+      } else {
+        while (r_iss > 0 && sW[r_iss - 1] >= z_near) --r_iss;
+      }
+      const int ngl = (H - r_iss + 7) >> 3;  // live groups of the nearest key
+#pragma unroll
+      for (int gi = 0; gi < NKS; ++gi) {
+        if (gi < ngl) {
+#pragma unroll
+          for (int i = 0; i < KB / 16; ++i) {
+            const int krow = i * 16 + (lane >> 1), half = lane & 1;
+            const int key = kb0 + krow;
+            const bool valid = key < m1;
+            const int keyc = valid ? key : m1 - 1;
+            const uint32_t off = gi * (KB * 32) + krow * 32 + ((half ^ ((krow >> 2) & 1)) << 4);
+            const int64_t tile = keyc / KT, kin = keyc % KT;
+            cp_async16(ks + off, Kb + ((tile * NKS + gi) * KT + kin) * 16 + half * 8, valid ? 16 : 0);
+          }
+        }
+      }
     }
   };
 
@@ -181,17 +221,6 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
     const int rq_far = MODE == ATF_MODE_COARSE ? (r_far >= H ? H : (r_far & ~7)) : r_far;
     const int rq_near = MODE == ATF_MODE_COARSE ? (r_near & ~7) : r_near;
     const bool uniform = rq_near == rq_far;
-    // K steps (16 pairs of one half) below the nearest key's first live pair are dead for every key
-    const int jl = rq_near >> 4;
-    // element masks of the K step that holds a first live pair r: lane t holds pairs 2t, 2t+1 of the
-    // step's first chunk and 8+2t, 9+2t of its second chunk
-    auto step_masks = [&](int r, uint32_t& mk0, uint32_t& mk1) {
-      const int e = r & 15;
-      mk0 = ((2 * t >= e) ? 0x0000FFFFu : 0u) | ((2 * t + 1 >= e) ? 0xFFFF0000u : 0u);
-      mk1 = ((8 + 2 * t >= e) ? 0x0000FFFFu : 0u) | ((9 + 2 * t >= e) ? 0xFFFF0000u : 0u);
-    };
-    uint32_t mku0 = 0xFFFFFFFFu, mku1 = 0xFFFFFFFFu;
-    if (uniform) step_masks(rq_far, mku0, mku1);
     // general blocks (the block straddles a window boundary): first live pair of this lane's key in each group
     int r_lane[NKG];
 #pragma unroll
@@ -205,49 +234,86 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
         r_lane[kg] = MODE == ATF_MODE_COARSE ? (r >= H ? H : (r & ~7)) : r;
       }
     }
-
-    // ---- S = q K^T ----
     float sc[NKG][4];
 #pragma unroll
     for (int kg = 0; kg < NKG; ++kg)
 #pragma unroll
       for (int e = 0; e < 4; ++e) sc[kg][e] = 0.f;
+
+    if (KL == ATF_KLAYOUT_ROWS) {
+      // ---- S = q K^T, row layout ----
+      // K steps (16 pairs of one half) below the nearest key's first live pair are dead for every key
+      const int jl = rq_near >> 4;
+      // element masks of the K step that holds a first live pair r: lane t holds pairs 2t, 2t+1 of the
+      // step's first chunk and 8+2t, 9+2t of its second chunk
+      auto step_masks = [&](int r, uint32_t& mk0, uint32_t& mk1) {
+        const int e = r & 15;
+        mk0 = ((2 * t >= e) ? 0x0000FFFFu : 0u) | ((2 * t + 1 >= e) ? 0xFFFF0000u : 0u);
+        mk1 = ((8 + 2 * t >= e) ? 0x0000FFFFu : 0u) | ((9 + 2 * t >= e) ? 0xFFFF0000u : 0u);
+      };
+      uint32_t mku0 = 0xFFFFFFFFu, mku1 = 0xFFFFFFFFu;
+      if (uniform) step_masks(rq_far, mku0, mku1);
 #pragma unroll
-    for (int j = 0; j < NKS; ++j) {
-      const int jh = j % (NKS / 2);  // K step within its half
-      if (jh < jl) continue;         // warp-uniform
+      for (int j = 0; j < NKS; ++j) {
+        const int jh = j % (NKS / 2);  // K step within its half
+        if (jh < jl) continue;         // warp-uniform
 #pragma unroll
-      for (int kp = 0; kp < NKG / 2; ++kp) {
-        // matrices: (group 2kp, chunk 2j), (group 2kp, chunk 2j+1), (group 2kp+1, chunk 2j), (group 2kp+1, chunk 2j+1)
-        const int mi = lane >> 3, mr = lane & 7;
-        const int row = (2 * kp + (mi >> 1)) * 8 + mr;
-        const int chunk = 2 * j + (mi & 1);
-        uint32_t bf[4];
-        ldsm_x4(ks + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
-        if (uniform) {
-          if (jh == (rq_far >> 4)) {
-            bf[0] &= mku0;
-            bf[1] &= mku1;
-            bf[2] &= mku0;
-            bf[3] &= mku1;
+        for (int kp = 0; kp < NKG / 2; ++kp) {
+          // matrices: (group 2kp, chunk 2j), (group 2kp, chunk 2j+1), (group 2kp+1, chunk 2j), (group 2kp+1, chunk 2j+1)
+          const int mi = lane >> 3, mr = lane & 7;
+          const int row = (2 * kp + (mi >> 1)) * 8 + mr;
+          const int chunk = 2 * j + (mi & 1);
+          uint32_t bf[4];
+          ldsm_x4(ks + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
+          if (uniform) {
+            if (jh == (rq_far >> 4)) {
+              bf[0] &= mku0;
+              bf[1] &= mku1;
+              bf[2] &= mku0;
+              bf[3] &= mku1;
+            }
+          } else {
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const int r = r_lane[2 * kp + h2];
+              uint32_t mk0 = 0xFFFFFFFFu, mk1 = 0xFFFFFFFFu;
+              if (jh < (r >> 4)) {
+                mk0 = 0u;
+                mk1 = 0u;
+              } else if (jh == (r >> 4)) {
+                step_masks(r, mk0, mk1);
+              }
+              bf[2 * h2] &= mk0;
+              bf[2 * h2 + 1] &= mk1;
+            }
           }
-        } else {
+          mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
+          mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
+        }
+      }
+    } else {
+      // ---- S = q K^T, group-major layout: K step j = the 8 pairs of group j; a key with first
+      //      live pair r keeps its first H - r pairs in this order ----
+      const int ngl = (H - rq_near + 7) >> 3;  // groups fetched for this block
+#pragma unroll
+      for (int j = 0; j < NKS; ++j) {
+        if (j >= ngl) continue;  // warp-uniform
+#pragma unroll
+        for (int kp = 0; kp < NKG / 2; ++kp) {
+          // matrices: (keys of group 2kp, first half), (same, second half), (keys of group 2kp+1, ...)
+          const int mi = lane >> 3, mr = lane & 7;
+          const int krow = (2 * kp + (mi >> 1)) * 8 + mr;
+          uint32_t bf[4];
+          ldsm_x4(ks + j * (KB * 32) + krow * 32 + (((mi & 1) ^ ((krow >> 2) & 1)) << 4), bf);
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
-            const int r = r_lane[2 * kp + h2];
-            uint32_t mk0 = 0xFFFFFFFFu, mk1 = 0xFFFFFFFFu;
-            if (jh < (r >> 4)) {
-              mk0 = 0u;
-              mk1 = 0u;
-            } else if (jh == (r >> 4)) {
-              step_masks(r, mk0, mk1);
-            }
-            bf[2 * h2] &= mk0;
-            bf[2 * h2 + 1] &= mk1;
+            const int live = H - r_lane[2 * kp + h2];  // pairs this lane's key keeps
+            if (8 * j + t >= live) bf[2 * h2] = 0u;
+            if (8 * j + 4 + t >= live) bf[2 * h2 + 1] = 0u;
           }
+          mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
+          mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
         }
-        mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
-        mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
       }
     }
     if (COUNT) {
@@ -408,12 +474,38 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   if (threadIdx.x == 0) P.counters[grp] = 0;  // ready for the next launch
 }
 
-template <int D>
+// K cache rows -> tiled group-major order [slab][tile][group][key in tile][16].  One thread per
+// (key, group of 8 pairs): gathers the 16 elements of the group (pair p = 8*group + i is dims
+// h-1-p and d-1-p) and writes 32 bytes.
+__global__ void __launch_bounds__(256)
+atf_kcache_pack_kernel(const __nv_bfloat16* __restrict__ K, __nv_bfloat16* __restrict__ Kg, int64_t slabs, int64_t n,
+                       int64_t ntiles, int64_t pos0, int D) {
+  const int H = D / 2, NG = D / 16;
+  const int64_t KT = (int64_t)DEC_WARPS * (DEC_TILE_BYTES / (D * 2));
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= slabs * n * NG) return;
+  const int gi = (int)(gid % NG);
+  const int64_t m = (gid / NG) % n, sl = gid / (NG * n);
+  const __nv_bfloat16* src = K + (sl * n + m) * D;
+  __align__(16) __nv_bfloat16 out[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = H - 1 - (8 * gi + i);
+    out[2 * i] = src[r];
+    out[2 * i + 1] = src[r + H];
+  }
+  const int64_t pos = pos0 + m, tile = pos / KT, kin = pos % KT;
+  uint4* dst = reinterpret_cast<uint4*>(Kg + (((sl * ntiles + tile) * NG + gi) * KT + kin) * 16);
+  dst[0] = reinterpret_cast<const uint4*>(out)[0];
+  dst[1] = reinterpret_cast<const uint4*>(out)[1];
+}
+
+template <int D, int KL>
 atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
   dim3 grid(P.nsplit, P.Hkv, B);
 #define ATF_DEC_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                  \
-    auto kern = atf_decode_kernel<D, MODE_, COUNT_>;                                                    \
+    auto kern = atf_decode_kernel<D, MODE_, COUNT_, KL>;                                                    \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DEC_SMEM));  \
     kern<<<grid, DEC_THREADS, DEC_SMEM, s>>>(P, t);                                                     \
   } while (0)
@@ -477,7 +569,7 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.G = Hq / Hkv;
   P.L = (int)L;
   P.nsplit = atf_decode_num_splits(B, Hkv, L);
-  const int kb = 2048 / d;  // keys per warp iteration
+  const int kb = DEC_WARPS * (2048 / d);  // keys per block iteration (one tile of the group-major cache)
   int64_t kps = (L + P.nsplit - 1) / P.nsplit;
   kps = (kps + kb - 1) / kb * kb;
   P.keys_per_split = (int)kps;
@@ -487,7 +579,31 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.partials = (float*)(base + ATF_WS_HEADER);
   cudaStream_t s = (cudaStream_t)stream;
   const bool count = P.kept != nullptr;
-  return d == 64 ? launch_decode<64>(P, t, B, mode, count, s) : launch_decode<128>(P, t, B, mode, count, s);
+  const int kl = opts ? opts->k_layout : ATF_KLAYOUT_ROWS;
+  if (kl != ATF_KLAYOUT_ROWS && kl != ATF_KLAYOUT_GROUPS) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: unknown k_layout %d", kl);
+  if (kl == ATF_KLAYOUT_ROWS)
+    return d == 64 ? launch_decode<64, ATF_KLAYOUT_ROWS>(P, t, B, mode, count, s)
+                   : launch_decode<128, ATF_KLAYOUT_ROWS>(P, t, B, mode, count, s);
+  return d == 64 ? launch_decode<64, ATF_KLAYOUT_GROUPS>(P, t, B, mode, count, s)
+                 : launch_decode<128, ATF_KLAYOUT_GROUPS>(P, t, B, mode, count, s);
+}
+
+extern "C" int64_t atf_kcache_tile_keys(int d) { return (d == 64 || d == 128) ? DEC_WARPS * (DEC_TILE_BYTES / (d * 2)) : 0; }
+
+extern "C" atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, int64_t n, int64_t Lcap, int64_t pos0,
+                                      int d, void* stream) {
+  if (!K || !Kg) return atf_fail(ATF_ERR_INVALID_ARG, "atf_kcache_pack: null pointer");
+  if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_kcache_pack: d must be 64 or 128 (got %d)", d);
+  if (B < 1 || Hkv < 1 || n < 1 || pos0 < 0 || pos0 + n > Lcap) return atf_fail(ATF_ERR_INVALID_ARG, "atf_kcache_pack: bad shape");
+  if (((uintptr_t)K | (uintptr_t)Kg) & 15) return atf_fail(ATF_ERR_INVALID_ARG, "atf_kcache_pack: pointers must be 16-byte aligned");
+  const int64_t total = (int64_t)B * Hkv * n * (d / 16);
+  const int64_t blocks = (total + 255) / 256;
+  if (blocks > 0x7FFFFFFF) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_kcache_pack: too large");
+  const int64_t kt = atf_kcache_tile_keys(d);
+  atf_kcache_pack_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+      (const __nv_bfloat16*)K, (__nv_bfloat16*)Kg, (int64_t)B * Hkv, n, (Lcap + kt - 1) / kt, pos0, d);
+  ATF_CUDA_CHECK(cudaGetLastError());
+  return ATF_OK;
 }
 
 extern "C" atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, void* O, int B, int Hq,

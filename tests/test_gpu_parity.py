@@ -151,6 +151,32 @@ def _decode_case(atf, w: gen.Workload, mode, table=None):
     # second call on the same workspace (split counters must have been reset)
     O2 = atf.atf_decode(q.cuda(), Kc.cuda(), Vc.cuda(), table=torch.from_numpy(Wo), mode=mode)
     assert torch.equal(O2, O)
+    # the same step from a group-major K cache: same terms, so the same counts and the same answer
+    Kg = atf.atf_kcache_pack(Kc.cuda())
+    kept.zero_()
+    O3, lse3 = atf.atf_decode(q.cuda(), Kg, Vc.cuda(), table=torch.from_numpy(Wo), mode=mode, kept_terms=kept,
+                              return_lse=True)
+    torch.cuda.synchronize()
+    _check_out(O3, lse3, Or, Lr, tag="group-major")
+    assert kept.cpu().tolist() == [want] * (w.B * w.Hq)
+
+
+def test_kcache_pack_layout(atf):
+    """Tile T, group j of the packed cache hold pairs r = h-1-8j-i (i = 0..7) of keys T*KT.. as (dim r, dim r+h)."""
+    B, Hkv, n, d = 2, 3, 150, 128
+    h, kt = d // 2, 64
+    K = gen.normal_bf16((B, Hkv, n, d), 123).cuda()
+    Kg = torch.zeros((B, Hkv, 3, d // 16, kt, 16), dtype=torch.bfloat16, device="cuda")
+    atf.atf_kcache_pack(K, Kg, pos0=5)
+    ref = torch.zeros_like(Kg)
+    for m in range(n):
+        pos = 5 + m
+        for j in range(d // 16):
+            for i in range(8):
+                r = h - 1 - (8 * j + i)
+                ref[:, :, pos // kt, j, pos % kt, 2 * i] = K[:, :, m, r]
+                ref[:, :, pos // kt, j, pos % kt, 2 * i + 1] = K[:, :, m, r + h]
+    assert torch.equal(Kg, ref)
 
 
 @pytest.mark.parametrize("mode", [0, 1])
