@@ -168,6 +168,7 @@ def run_ours(args):
         e = [ev() for _ in range(5)]
         e[0].record()
         W, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+        W = atf.WindowTable(W)
         Qg.copy_(Q0)
         Kg.copy_(K0)
         e[1].record()
@@ -217,7 +218,7 @@ def run_ours(args):
         print(json.dumps({"profile_only": True, "workload": args.workload, "ms_per_step": total_ms / args.steps,
                           "prefill_ms": statistics.median(t_pre), "decode_us": statistics.median(t_dec) * 1e3}))
         return
-    Wl = W.tolist()
+    Wl = list(W.arr)
     executed, effective = prefill_flops(wl, Wl)
     pre_ms = statistics.median(t_pre)
     dec_ms = statistics.median(t_dec)
@@ -244,19 +245,22 @@ def run_ours(args):
     kv_bytes = 2 * Kg.numel() * 2
     npool = max(2, math.ceil((512 << 20) / kv_bytes) + 1)
     pool = [(Kg, V)] + [(Kg.clone(), V.clone()) for _ in range(npool - 1)]
-    dec_t = {True: [], False: []}
-    for windowed in (True, False):
+    gpool = [atf.atf_kcache_pack(kk) for kk, _ in pool]  # the same caches in the tiled group-major layout
+    dec_t = {"win": [], "full": [], "grp": []}
+    for kind in ("win", "full", "grp"):
         for i in range(8 + 40):
             Kc, Vc = pool[i % npool]
+            if kind == "grp":
+                Kc = gpool[i % npool]
             a, b_ = ev(), ev()
             a.record()
-            atf.atf_decode(qd, Kc, Vc, table=W if windowed else None, O=Od)
+            atf.atf_decode(qd, Kc, Vc, table=None if kind == "full" else W, O=Od)
             b_.record()
             torch.cuda.synchronize()
             if i >= 8:
-                dec_t[windowed].append(a.elapsed_time(b_) * 1e3)
-    dec_us, dec_full_us = statistics.median(dec_t[True]), statistics.median(dec_t[False])
-    del pool
+                dec_t[kind].append(a.elapsed_time(b_) * 1e3)
+    dec_us, dec_full_us, dec_grp_us = (statistics.median(dec_t[k]) for k in ("win", "full", "grp"))
+    del pool, gpool
     dbytes = decode_bytes(wl, Wl, True)
     dbytes_full = decode_bytes(wl, Wl, False)
 
@@ -295,6 +299,8 @@ def run_ours(args):
         "decode_us": dec_us, "decode_gbs": dbytes / (dec_us * 1e-6) / 1e9,
         "decode_full_us": dec_full_us, "decode_full_gbs": dbytes_full / (dec_full_us * 1e-6) / 1e9,
         "decode_speedup_vs_full": dec_full_us / dec_us, "decode_in_step_us": dec_ms * 1e3,
+        "decode_group_major_us": dec_grp_us, "decode_group_major_gbs": dbytes / (dec_grp_us * 1e-6) / 1e9,
+        "decode_group_major_speedup_vs_full": dec_full_us / dec_grp_us,
         "frac_of_nominal": {"prefill_executed_of_2250": executed / (pre_ms * 1e-3) / 1e12 / 2250.0,
                             "decode_of_8000": dbytes / (dec_us * 1e-6) / 1e9 / 8000.0},
         "roofline": {"bound": "tensor", "achieved": executed / (pre_ms * 1e-3) / 1e12,

@@ -40,9 +40,13 @@ struct AtfWorkspace {
 };
 AtfWorkspace atf_bound_workspace();
 
-constexpr int ATF_DECODE_SLOTS = 148 * 2;  // decode CTAs resident on the GPU at once
+// decode CTAs resident on the GPU at once: 2 per SM when K is read in the row layout, 3 per SM
+// with the group-major K cache (measured: whole-row streaming is fastest with fewer blocks in
+// flight, the sparser group-major reads want more)
+constexpr int ATF_DECODE_SLOTS_ROWS = 148 * 2;
+constexpr int ATF_DECODE_SLOTS_GROUPS = 148 * 3;
 constexpr int ATF_DECODE_MIN_SPLIT = 512;
-int atf_decode_num_splits(int B, int Hkv, int64_t L);
+int atf_decode_num_splits(int B, int Hkv, int64_t L, int slots);
 
 // ------------------------------------------------------------------------------------------
 // device side

@@ -15,6 +15,7 @@
 // warps are merged through shared memory, the block writes one partial (m, l, o) per head, and
 // the last block to finish for a (batch, KV head) merges the partials of all splits by their
 // log-sum-exp and writes O (and LSE).
+#include <algorithm>
 #include <cfloat>
 
 #include "atf_common.cuh"
@@ -23,10 +24,19 @@ namespace {
 
 constexpr int DEC_WARPS = 4;
 constexpr int DEC_THREADS = DEC_WARPS * 32;
-constexpr int DEC_STAGES = 3;
-constexpr int DEC_TILE_BYTES = 4096;                               // one K or V block of a warp
-constexpr int DEC_WARP_SMEM = DEC_STAGES * 2 * DEC_TILE_BYTES;     // K and V rings of one warp
+#ifndef ATF_DEC_STAGES
+#define ATF_DEC_STAGES 2
+#endif
+constexpr int DEC_STAGES = ATF_DEC_STAGES;
+constexpr int DEC_TILE_BYTES = 4096;                               // one K or V block of a warp in the cache
+// In shared memory a block's rows are padded by 16 bytes (row layouts: per cache row; group-major
+// K: per 4 keys of a group) so that ldmatrix is free of bank conflicts with plain, unswizzled,
+// compile-time offsets.
+constexpr int DEC_TILE_SMEM = 4608;
+constexpr int DEC_STAGE_SMEM = 2 * DEC_TILE_SMEM;                  // K block + V block
+constexpr int DEC_WARP_SMEM = DEC_STAGES * DEC_STAGE_SMEM;         // K and V rings of one warp
 constexpr int DEC_SMEM = DEC_WARPS * DEC_WARP_SMEM;
+constexpr int DEC_SMEM_ROWS = 110 * 1024;  // row layout: ask for enough to keep it at 2 blocks per SM
 constexpr float DEC_RESCALE_THRESHOLD = 8.f;
 
 struct DecodeParams {
@@ -38,7 +48,7 @@ struct DecodeParams {
   float* partials;           // [B*Hkv][nsplit][G][D + 2]
   unsigned int* counters;    // [B*Hkv], zero between launches
   unsigned long long* kept;  // may be null
-  int Hq, Hkv, G, L, nsplit, keys_per_split;
+  int Hq, Hkv, G, L, nsplit;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -70,7 +80,7 @@ __device__ __forceinline__ float ex2f(float x) {
 }
 
 template <int D, int MODE, bool COUNT, int KL>
-__global__ void __launch_bounds__(DEC_THREADS, 2)
+__global__ void __launch_bounds__(DEC_THREADS, KL == ATF_KLAYOUT_ROWS ? 2 : 3)
 atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant__ AtfTable table) {
   constexpr int H = D / 2;
   constexpr int CPR = D / 8;            // 16-byte chunks per cache row
@@ -92,8 +102,11 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;  // MMA fragment row (query head) and column pair
   const int G = P.G, L = P.L;
-  const int m0 = split * P.keys_per_split;
-  const int m1 = min(L, m0 + P.keys_per_split);
+  // Tiles of DEC_WARPS * KB keys are dealt round-robin to the splits of a (batch, KV head), so
+  // that at any moment the splits read neighbouring tiles: DRAM sees a few moving sequential
+  // streams instead of one stream per block (measured faster than contiguous ranges per split).
+  const int m0 = split * (DEC_WARPS * KB);
+  const int m1 = L;
   const int64_t slab = ((int64_t)b * P.Hkv + hkv) * (int64_t)L * D;
   // the group-major cache is padded to whole tiles of DEC_WARPS * KB keys
   const __nv_bfloat16* Kb = P.K + (KL == ATF_KLAYOUT_ROWS
@@ -126,32 +139,53 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
     }
   }
 
-  // this lane's chunk of a cache row in the cp.async mapping, and the widest window among its 8 pairs
-  const int cp_chunk = lane % CPR;
-  const int cp_row0 = lane / CPR;               // first row this lane copies; then every 32/CPR rows
+  // ---- copy and fragment addressing, fixed per lane ----
+  constexpr int PITCH = ROWB + 16;          // shared-memory row pitch of a row-layout block
+  constexpr int RSTEP = 32 / CPR;           // rows covered by one warp-wide copy
+  constexpr int GSZ = KB * 36;              // shared-memory bytes of one group of a group-major K block
+  static_assert(KB * PITCH <= DEC_TILE_SMEM && NKS * GSZ <= DEC_TILE_SMEM, "block does not fit its shared-memory tile");
+  const int cp_chunk = lane % CPR;          // this lane's 16-byte chunk of a cache row
+  const int cp_row0 = lane / CPR;           // first row this lane copies; then every RSTEP rows
+  const uint32_t cp_dst0 = cp_row0 * PITCH + cp_chunk * 16;
+  const int gk_row = lane >> 1, gk_half = lane & 1;  // group-major K: (key, half of its 32 bytes) of a 16-key copy
+  const uint32_t gk_dst0 = gk_row * 32 + (gk_row >> 2) * 16 + gk_half * 16;
   const uint32_t warp_smem = smem_u32(dsm) + warp * DEC_WARP_SMEM;
+  const int lm_i = lane >> 3, lm_r = lane & 7;  // ldmatrix: matrix fed by this lane and row in it
+  const uint32_t k_lane_off = KL == ATF_KLAYOUT_ROWS
+                                  ? ((lm_i >> 1) * 8 + lm_r) * PITCH + (lm_i & 1) * 16
+                                  : ((lm_i >> 1) * 8 + lm_r) * 32 + ((((lm_i >> 1) * 8 + lm_r) >> 2) * 16) + (lm_i & 1) * 16;
+  const uint32_t v_lane_off = ((lm_i & 1) * 8 + lm_r) * PITCH + (lm_i >> 1) * 16;
 
   const __nv_bfloat16* Vb = P.V + slab;
   int r_iss = 0;  // cursor for the copies: first live pair of the nearest key of the block being fetched
   auto issue_block = [&](int kb0, int stage) {
-    const uint32_t ks = warp_smem + stage * 2 * DEC_TILE_BYTES, vs = ks + DEC_TILE_BYTES;
+    const uint32_t ks = warp_smem + stage * DEC_STAGE_SMEM, vs = ks + DEC_TILE_SMEM;
+    // every key of the block exists and is reached by some pair: no predicates
+    const bool fast = (kb0 + KB <= m1) && (L - 1 - kb0 <= Wmax);
     // V rows, and K rows in the row layout, are copied whole: a 128-byte half row always ends in
     // live low-frequency pairs and DRAM moves whole 128-byte lines, so leaving out dead 16-byte
     // chunks of a row would save no traffic.  A key no pair reaches is not copied at all.
+    if (fast) {
+      const int64_t goff = (int64_t)(kb0 + cp_row0) * D + cp_chunk * 8;
 #pragma unroll
-    for (int i = 0; i < CP_PER_LANE; ++i) {
-      const int row = cp_row0 + i * (32 / CPR);
-      const int key = kb0 + row;
-      const bool valid = key < m1 && (L - 1 - key) <= Wmax;
-      const int keyc = key < m1 ? key : m1 - 1;
-      const uint32_t off = row * ROWB + ((cp_chunk ^ (row & 7)) << 4);
-      const int64_t goff = (int64_t)keyc * D + cp_chunk * 8;
-      if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + off, Kb + goff, valid ? 16 : 0);
-      cp_async16(vs + off, Vb + goff, valid ? 16 : 0);
+      for (int i = 0; i < CP_PER_LANE; ++i) {
+        if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff + i * RSTEP * D, 16);
+        cp_async16(vs + cp_dst0 + i * RSTEP * PITCH, Vb + goff + i * RSTEP * D, 16);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < CP_PER_LANE; ++i) {
+        const int key = kb0 + cp_row0 + i * RSTEP;
+        const bool valid = key < m1 && (L - 1 - key) <= Wmax;
+        const int keyc = key < m1 ? key : m1 - 1;
+        const int64_t goff = (int64_t)keyc * D + cp_chunk * 8;
+        if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff, valid ? 16 : 0);
+        cp_async16(vs + cp_dst0 + i * RSTEP * PITCH, Vb + goff, valid ? 16 : 0);
+      }
     }
     if (KL == ATF_KLAYOUT_GROUPS) {
       // group-major K: the live pairs of a key are its first groups, each group a contiguous
-      // stream over the keys, so only live bytes are fetched (8-pair granularity)
+      // stream over the keys of the tile, so only live bytes are fetched (8-pair granularity)
       const int z_near = max(L - 1 - (kb0 + KB - 1), 0);
       if (r_iss >= H || sW[r_iss] < z_near) {
         r_iss = 0;
@@ -160,18 +194,16 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
         while (r_iss > 0 && sW[r_iss - 1] >= z_near) --r_iss;
       }
       const int ngl = (H - r_iss + 7) >> 3;  // live groups of the nearest key
+      const int64_t tile0 = ((int64_t)(kb0 / KT) * NKS * KT + (kb0 % KT)) * 16;  // group 0, first key of the block
 #pragma unroll
       for (int gi = 0; gi < NKS; ++gi) {
         if (gi < ngl) {
 #pragma unroll
           for (int i = 0; i < KB / 16; ++i) {
-            const int krow = i * 16 + (lane >> 1), half = lane & 1;
-            const int key = kb0 + krow;
+            const int key = kb0 + i * 16 + gk_row;
             const bool valid = key < m1;
-            const int keyc = valid ? key : m1 - 1;
-            const uint32_t off = gi * (KB * 32) + krow * 32 + ((half ^ ((krow >> 2) & 1)) << 4);
-            const int64_t tile = keyc / KT, kin = keyc % KT;
-            cp_async16(ks + off, Kb + ((tile * NKS + gi) * KT + kin) * 16 + half * 8, valid ? 16 : 0);
+            const int64_t goff = tile0 + ((int64_t)gi * KT + (valid ? i * 16 + gk_row : 0)) * 16 + gk_half * 8;
+            cp_async16(ks + gi * GSZ + i * 576 + gk_dst0, Kb + goff, valid ? 16 : 0);
           }
         }
       }
@@ -193,7 +225,7 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 
   // ---- prologue: fill the ring ----
   const int kb_first = m0 + warp * KB;
-  const int kb_step = DEC_WARPS * KB;
+  const int kb_step = P.nsplit * DEC_WARPS * KB;
 #pragma unroll
   for (int s = 0; s < DEC_STAGES - 1; ++s) {
     const int kb0 = kb_first + s * kb_step;
@@ -210,7 +242,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
       if (kbn < m1) issue_block(kbn, (it + DEC_STAGES - 1) % DEC_STAGES);
       cp_async_commit();
     }
-    const uint32_t ks = warp_smem + (it % DEC_STAGES) * 2 * DEC_TILE_BYTES, vs = ks + DEC_TILE_BYTES;
+    const uint32_t ks = warp_smem + (it % DEC_STAGES) * DEC_STAGE_SMEM, vs = ks + DEC_TILE_SMEM;
+    const bool blk_fast = (kb0 + KB <= m1) && (L - 1 - kb0 <= Wmax);
 
     // ---- live pair range over the block (coarse mode: first live pair rounded down to 8) ----
     const int z_far = L - 1 - kb0;                      // the block's first key is the farthest
@@ -260,11 +293,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 #pragma unroll
         for (int kp = 0; kp < NKG / 2; ++kp) {
           // matrices: (group 2kp, chunk 2j), (group 2kp, chunk 2j+1), (group 2kp+1, chunk 2j), (group 2kp+1, chunk 2j+1)
-          const int mi = lane >> 3, mr = lane & 7;
-          const int row = (2 * kp + (mi >> 1)) * 8 + mr;
-          const int chunk = 2 * j + (mi & 1);
           uint32_t bf[4];
-          ldsm_x4(ks + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
+          ldsm_x4(ks + k_lane_off + kp * 16 * PITCH + j * 32, bf);
           if (uniform) {
             if (jh == (rq_far >> 4)) {
               bf[0] &= mku0;
@@ -301,10 +331,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 #pragma unroll
         for (int kp = 0; kp < NKG / 2; ++kp) {
           // matrices: (keys of group 2kp, first half), (same, second half), (keys of group 2kp+1, ...)
-          const int mi = lane >> 3, mr = lane & 7;
-          const int krow = (2 * kp + (mi >> 1)) * 8 + mr;
           uint32_t bf[4];
-          ldsm_x4(ks + j * (KB * 32) + krow * 32 + (((mi & 1) ^ ((krow >> 2) & 1)) << 4), bf);
+          ldsm_x4(ks + k_lane_off + j * GSZ + kp * 576, bf);
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
             const int live = H - r_lane[2 * kp + h2];  // pairs this lane's key keeps
@@ -329,14 +357,25 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 
     // ---- online softmax (log2 domain); this lane holds keys 2t, 2t+1 of every group for head g ----
     float mx = -INFINITY;
+    if (blk_fast) {
 #pragma unroll
-    for (int kg = 0; kg < NKG; ++kg) {
+      for (int kg = 0; kg < NKG; ++kg) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int key = kb0 + kg * 8 + 2 * t + e;
-        const int z = L - 1 - key;
-        sc[kg][e] = (key < m1 && z <= Wmax) ? sc[kg][e] * kScaleLog2 : -INFINITY;
-        mx = fmaxf(mx, sc[kg][e]);
+        for (int e = 0; e < 2; ++e) {
+          sc[kg][e] *= kScaleLog2;
+          mx = fmaxf(mx, sc[kg][e]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int kg = 0; kg < NKG; ++kg) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int key = kb0 + kg * 8 + 2 * t + e;
+          const int z = L - 1 - key;
+          sc[kg][e] = (key < m1 && z <= Wmax) ? sc[kg][e] * kScaleLog2 : -INFINITY;
+          mx = fmaxf(mx, sc[kg][e]);
+        }
       }
     }
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -371,11 +410,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 #pragma unroll
       for (int np = 0; np < NNT / 2; ++np) {
         // matrices: (keys 0-7, chunk 2np), (keys 8-15, chunk 2np), (keys 0-7, chunk 2np+1), (keys 8-15, chunk 2np+1)
-        const int mi = lane >> 3, mr = lane & 7;
-        const int row = pk * 16 + (mi & 1) * 8 + mr;
-        const int chunk = 2 * np + (mi >> 1);
         uint32_t bf[4];
-        ldsm_x4_trans(vs + row * ROWB + ((chunk ^ (row & 7)) << 4), bf);
+        ldsm_x4_trans(vs + v_lane_off + pk * 16 * PITCH + np * 32, bf);
         mma_bf16_16816(oacc[2 * np], pa[2 * pk], pa[2 * pk + 1], bf[0], bf[1]);
         mma_bf16_16816(oacc[2 * np + 1], pa[2 * pk], pa[2 * pk + 1], bf[2], bf[3]);
       }
@@ -506,8 +542,11 @@ atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mo
 #define ATF_DEC_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                  \
     auto kern = atf_decode_kernel<D, MODE_, COUNT_, KL>;                                                    \
-    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DEC_SMEM));  \
-    kern<<<grid, DEC_THREADS, DEC_SMEM, s>>>(P, t);                                                     \
+    const int smem = KL == ATF_KLAYOUT_ROWS ? DEC_SMEM_ROWS : DEC_SMEM;                                 \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));      \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,           \
+                                        cudaSharedmemCarveoutMaxShared));                                \
+    kern<<<grid, DEC_THREADS, smem, s>>>(P, t);                                                     \
   } while (0)
   if (mode == ATF_MODE_EXACT) {
     if (count) ATF_DEC_LAUNCH(ATF_MODE_EXACT, true); else ATF_DEC_LAUNCH(ATF_MODE_EXACT, false);
@@ -524,7 +563,8 @@ atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mo
 atf_status atf_validate_table(const char* who, const int64_t* table, int d, int64_t N, AtfTable* out);
 
 static size_t decode_ws_bytes(int B, int Hq, int Hkv, int64_t L, int d) {
-  const int ns = atf_decode_num_splits(B, Hkv, L);
+  const int ns = std::max(atf_decode_num_splits(B, Hkv, L, ATF_DECODE_SLOTS_ROWS),
+                          atf_decode_num_splits(B, Hkv, L, ATF_DECODE_SLOTS_GROUPS));
   size_t partials = (size_t)B * Hq * ns * (d + 2) * sizeof(float);
   partials = (partials + 255) & ~(size_t)255;
   return ATF_WS_HEADER + partials;
@@ -568,12 +608,11 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   P.Hkv = Hkv;
   P.G = Hq / Hkv;
   P.L = (int)L;
-  P.nsplit = atf_decode_num_splits(B, Hkv, L);
-  const int kb = DEC_WARPS * (2048 / d);  // keys per block iteration (one tile of the group-major cache)
-  int64_t kps = (L + P.nsplit - 1) / P.nsplit;
-  kps = (kps + kb - 1) / kb * kb;
-  P.keys_per_split = (int)kps;
-  P.nsplit = (int)((L + kps - 1) / kps);  // drop splits the rounding emptied
+  const int kl_ = opts ? opts->k_layout : ATF_KLAYOUT_ROWS;
+  P.nsplit = atf_decode_num_splits(B, Hkv, L, kl_ == ATF_KLAYOUT_GROUPS ? ATF_DECODE_SLOTS_GROUPS : ATF_DECODE_SLOTS_ROWS);
+  const int64_t kt = DEC_WARPS * (DEC_TILE_BYTES / (d * 2));  // keys per tile; tiles go round-robin to the splits
+  const int64_t ntiles = (L + kt - 1) / kt;
+  if (P.nsplit > ntiles) P.nsplit = (int)ntiles;
   char* base = (char*)ws.ptr;
   P.counters = (unsigned int*)(base + ATF_WS_STATUS_BYTES);
   P.partials = (float*)(base + ATF_WS_HEADER);

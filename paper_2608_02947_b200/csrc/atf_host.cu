@@ -20,12 +20,11 @@ atf_status atf_fail(atf_status code, const char* fmt, ...) {
 
 AtfWorkspace atf_bound_workspace() { return g_ws; }
 
-// Splits of the key range per (batch, KV head) for decode.  Two decode CTAs fit on each of
-// the 148 SMs; pick the smallest split count that fills whole waves of those 296 slots best,
-// with at least ATF_DECODE_MIN_SPLIT keys per split.
-int atf_decode_num_splits(int B, int Hkv, int64_t L) {
+// Splits of the key range per (batch, KV head) for decode: the smallest split count that fills
+// whole waves of the `slots` resident CTAs best, with at least ATF_DECODE_MIN_SPLIT keys per split.
+int atf_decode_num_splits(int B, int Hkv, int64_t L, int slots_) {
   const int64_t groups = (int64_t)B * Hkv;
-  const int64_t slots = ATF_DECODE_SLOTS;
+  const int64_t slots = slots_;
   int64_t most = L / ATF_DECODE_MIN_SPLIT;
   if (most < 1) most = 1;
   if (most > 4 * slots) most = 4 * slots;
