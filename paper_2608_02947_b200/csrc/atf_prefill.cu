@@ -106,16 +106,20 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
 // span distances [zmin, zmax].  w[] is non-decreasing, so the pairs reaching a distance z are
 // r >= r0(z), and r0 only grows with dt: the cursors are advanced, never rewound.
 struct TileSched {
-  // first pair live in some cell / in most cells (window reaches the tile's central distance)
-  // / in every cell of the tile
+  // For the 32 query rows of softmax warp wq (0..3) of a tile at tile distance dt, the cells span
+  // distances [zlo, zhi].  r_any / r_all: first pair live in some / in every one of those cells.
+  // r_mid: first pair kept in the MMA for those rows, i.e. live at the distance from the warp's
+  // middle row to the tile's middle column (live in most of the warp's cells).  A pair kept by
+  // warp 0 (the rows nearest to the keys) is in the MMA depth of the whole tile; the rows of the
+  // other warps that do not keep it hold a zero in that column of Q.
   int r_any = 0, r_mid = 0, r_all = 0;
-  __device__ __forceinline__ void advance(const int* w, int H, int dt) {
-    const int zmin = dt == 0 ? 0 : (dt - 1) * T + 1;
-    const int zmid = dt == 0 ? T / 2 : dt * T;
-    const int zmax = (dt + 1) * T - 1;
-    while (r_any < H && w[r_any] < zmin) ++r_any;
+  __device__ __forceinline__ void advance(const int* w, int H, int dt, int wq) {
+    const int zlo = dt == 0 ? 0 : dt * T + 32 * wq - (T - 1);
+    const int zhi = dt * T + 32 * wq + 31;
+    const int zmid = dt == 0 ? 16 * wq + 15 : dt * T + 32 * wq - 48;
+    while (r_any < H && w[r_any] < zlo) ++r_any;
     while (r_mid < H && w[r_mid] < zmid) ++r_mid;
-    while (r_all < H && w[r_all] < zmax) ++r_all;
+    while (r_all < H && w[r_all] < zhi) ++r_all;
   }
 };
 // Pairs contracted by the MMA for a tile.  Exact mode: the pairs live in most cells (the few
@@ -256,7 +260,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       for (int t = 0; t < Tt; ++t) {
         const int j = itB - t;
         const int dnear = max(t - 1, 0);  // the closer user of this key tile
-        sc.advance(sW, H, dnear);
+        sc.advance(sW, H, dnear, 0);
         const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, dnear);
         const int ncols = MODE == ATF_MODE_EXACT ? 2 * (H - sc.r_any) : 2 * depth;
         const int nkb = max(1, (ncols + 63) / 64);
@@ -287,7 +291,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
       auto issue_qk = [&](int X, int v, int tile) {
         TileSched& sc = X ? scB : scA;
-        sc.advance(sW, H, v);
+        sc.advance(sW, H, v, 0);
         const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, v);
         const int natoms = (depth + 7) / 8;
         const uint64_t q0 = X ? dQ1 : dQ0, k0 = (tile & 1) ? dK1 : dK0;
@@ -368,6 +372,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
     if (!ok) fail_site = 30;
+    // exact mode keeps/zeroes pairs per warp of rows; coarse mode decides per tile (warp 0's view)
+    const int wq = MODE == ATF_MODE_EXACT ? (warp & 3) : 0;
     TileSched sc;
     int zeroed_from = H;  // pairs p >= zeroed_from are zero in the shared copy of Q_X
     auto zero_q_down_to = [&](int p_keep) {
@@ -382,7 +388,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     };
     if (ok) {
-      sc.advance(sW, H, 0);
+      sc.advance(sW, H, 0, wq);
       zero_q_down_to(H - sc.r_mid);
       mbar_arrive(bar(B_QZ + X));
     }
@@ -434,34 +440,54 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         //      no row of this warp has such a cell in it. ----
         if (MODE == ATF_MODE_EXACT) {
           const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
+          const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
+          uint32_t qq_next = (p_all < p_any) ? *reinterpret_cast<const uint32_t*>(qsrc + 2 * p_all) : 0u;
           for (int p = p_all; p < p_any; ++p) {
             const int wp = sW[H - 1 - p];
             const bool subtract = p < p_mid;
-            float q0 = 0.f, q1 = 0.f;
-            if (row_ok) {
-              const uint32_t qq = *reinterpret_cast<const uint32_t*>(P.Qp + ((int64_t)bhq * P.N + n) * D + 2 * p);
-              q0 = bf16lo_to_f32(qq);
-              q1 = bf16hi_to_f32(qq);
-            }
+            const uint32_t qq = qq_next;
+#ifndef ATF_EXP_NOQ
+            if (p + 1 < p_any) qq_next = *reinterpret_cast<const uint32_t*>(qsrc + 2 * (p + 1));  // overlaps this pair's work
+#endif
+            float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
             if (subtract) {
               q0 = -q0;
               q1 = -q1;
             }
             const int col = 2 * p;
-            const uint8_t* kbase = smem_gen + SM::K_OFF + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+            // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
+            const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
             const int chunk = (col & 63) >> 3;
-  #pragma unroll
+            uint32_t base8[8];
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
+            // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
+            // is formed on the FMA pipe as a saturated affine function of its column (the integer and
+            // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
+            const float jbf = (float)(zrow - wp);
+            const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
+#pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
               // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
               const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
+#ifdef ATF_TRACE
+              if (touched && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[15 * 64 + v] += 1;
+              if (q4 == 0 && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[4 * 64 + v] += 1;
+#endif
               if (touched) {
-  #pragma unroll
+                // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
+                uint32_t kk[32];
+#pragma unroll
                 for (int cc = 0; cc < 32; ++cc) {
                   const int c = q4 * 32 + cc;
-                  const uint32_t kk = *reinterpret_cast<const uint32_t*>(kbase + c * 128 + ((chunk ^ (c & 7)) << 4));
-                  const float term = fmaf(q0, bf16lo_to_f32(kk), q1 * bf16hi_to_f32(kk));
-                  const bool inside = zrow - c <= wp;
-                  s[c] += (inside != subtract) ? term : 0.f;
+                  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + c * 128));
+                }
+#pragma unroll
+                for (int cc = 0; cc < 32; ++cc) {
+                  const int c = q4 * 32 + cc;
+                  const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
+                  const float coef = __saturatef(fmaf(ca, (float)c, cb));
+                  s[c] = fmaf(term, coef, s[c]);
                 }
               }
             }
@@ -546,7 +572,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       tc_st32(tS + 32, pk + 32);
       // zero the Q columns that stop being live in most cells at the next step
       if (v + 1 < nX) {
-        sc.advance(sW, H, dt + 1);
+        sc.advance(sW, H, dt + 1, wq);
         zero_q_down_to(H - sc.r_mid);
       }
       tc_wait_st();
