@@ -289,26 +289,81 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const uint64_t dV0 = make_smem_desc_sw128(sV, BLK_BYTES, 1024),
                      dV1 = make_smem_desc_sw128(sV + SM::TILE, BLK_BYTES, 1024);
       // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
-      auto issue_qk = [&](int X, int v, int tile) {
+      // live depth (in 16-column MMA steps) of step v of tile X; computed ahead of time, while the
+      // issuer would otherwise be waiting, because a lone thread runs such code slowly
+      auto depth_atoms = [&](int X, int v) {
         TileSched& sc = X ? scB : scA;
         sc.advance(sW, H, v, 0);
-        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, v);
-        const int natoms = (depth + 7) / 8;
-        const uint64_t q0 = X ? dQ1 : dQ0, k0 = (tile & 1) ? dK1 : dK0;
-        const uint32_t d = tmem_base + X * T;
-#pragma unroll
-        for (int a = 0; a < D / 16; ++a) {
-          const uint64_t off = (uint64_t)(((a >> 2) * BLK_BYTES + (a & 3) * 32) >> 4);
-          if (a < natoms) tc_mma_ss(d, q0 + off, k0 + off, IDESC_QK, a > 0 ? 1u : 0u);
-        }
+        return (tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, v) + 7) / 8;
+      };
+      int natomsA = depth_atoms(0, 0), natomsB = depth_atoms(1, 0);
+      auto issue_qk = [&](int X, int v, int tile) {
+        const int natoms = X ? natomsB : natomsA;
+        const uint64_t dQ = X ? dQ1 : dQ0, k0 = (tile & 1) ? dK1 : dK0;
+        const uint32_t tSx = tmem_base + X * T;
+        if (X == 1) ATF_STAMP(13, v - 1);
+        asm volatile(
+            "{\n\t"
+            ".reg .pred pf, p0, p1, p2, p3, p4, p5, p6, p7;\n\t"
+            ".reg .b64 qd, kd;\n\t"
+            "setp.eq.u32 pf, %4, 0xffffffff;\n\t"  // false: the first step overwrites S
+            "setp.gt.u32 p0, %4, 0;\n\t"
+            "setp.gt.u32 p1, %4, 1;\n\t"
+            "setp.gt.u32 p2, %4, 2;\n\t"
+            "setp.gt.u32 p3, %4, 3;\n\t"
+            "setp.gt.u32 p4, %4, 4;\n\t"
+            "setp.gt.u32 p5, %4, 5;\n\t"
+            "setp.gt.u32 p6, %4, 6;\n\t"
+            "setp.gt.u32 p7, %4, 7;\n\t"
+            "@p0 tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+            "add.u64 qd, %1, 2;\n\t add.u64 kd, %2, 2;\n\t"
+            "@p1 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 4;\n\t add.u64 kd, %2, 4;\n\t"
+            "@p2 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 6;\n\t add.u64 kd, %2, 6;\n\t"
+            "@p3 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 1024;\n\t add.u64 kd, %2, 1024;\n\t"
+            "@p4 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 1026;\n\t add.u64 kd, %2, 1026;\n\t"
+            "@p5 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 1028;\n\t add.u64 kd, %2, 1028;\n\t"
+            "@p6 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "add.u64 qd, %1, 1030;\n\t add.u64 kd, %2, 1030;\n\t"
+            "@p7 tcgen05.mma.cta_group::1.kind::f16 [%0], qd, kd, %3, p0;\n\t"
+            "}"
+            ::"r"(tSx), "l"(dQ), "l"(k0), "r"(IDESC_QK), "r"((uint32_t)natoms)
+            : "memory");
+        if (X == 1) ATF_STAMP(14, v - 1);
         tc_commit(bar(B_SFULL + X));
       };
       auto issue_pv = [&](int X, int v, int tile) {
         const uint64_t v0 = (tile & 1) ? dV1 : dV0;
-        const uint32_t d = tmem_base + 2 * T + X * D, p = tmem_base + X * T;
-        tc_mma_ts(d, p, v0, IDESC_PV, v == 0 ? 0u : 1u);
-#pragma unroll
-        for (int ks = 1; ks < T / 16; ++ks) tc_mma_ts(d, p + ks * 8, v0 + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
+        const uint32_t tOx = tmem_base + 2 * T + X * D, tSx = tmem_base + X * T;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred pf, pt;\n\t"
+            ".reg .b64 vd;\n\t"
+            ".reg .b32 pa;\n\t"
+            "setp.ne.b32 pf, %4, 0;\n\t"  // the very first step of the tile overwrites O
+            "setp.eq.u32 pt, %4, %4;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n\t"
+            "add.u32 pa, %1, 8;\n\t add.u64 vd, %2, 128;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 16;\n\t add.u64 vd, %2, 256;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 24;\n\t add.u64 vd, %2, 384;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 32;\n\t add.u64 vd, %2, 512;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 40;\n\t add.u64 vd, %2, 640;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 48;\n\t add.u64 vd, %2, 768;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "add.u32 pa, %1, 56;\n\t add.u64 vd, %2, 896;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
+            "}"
+            ::"r"(tOx), "r"(tSx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)v)
+            : "memory");
       };
       bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
       if (!ok) fail_site = 20;
@@ -328,6 +383,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (pvB || pvA) ok = ok && wait_or_abort(bar(B_VFULL + s % VS), (s / VS) & 1, abortp);
         if (qkB || qkA) ok = ok && wait_or_abort(bar(B_KFULL + (s + 1) % KS), ((s + 1) / KS) & 1, abortp);
         if (!ok) { fail_site = 22; break; }
+        if (qkB) natomsB = depth_atoms(1, s + 1);
         if (pvB) {
           if (!wait_or_abort(bar(B_PFULL + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
           tc_fence_after();
@@ -338,10 +394,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (qkB) issue_qk(1, s + 1, s + 1);
         else if (pvB) tc_commit(bar(B_OFULL + 1));
         ATF_STAMP(12, s);
+        if (qkA && s > 0) natomsA = depth_atoms(0, s);
         if (pvA) {
           if (!wait_or_abort(bar(B_PFULL + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
           tc_fence_after();
-          ATF_STAMP(13, s);
           issue_pv(0, s - 1, s);
         }
         if (qkA) {
@@ -351,7 +407,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         } else if (pvA) {
           tc_commit(bar(B_OFULL + 0));
         }
-        ATF_STAMP(14, s);
         if (s + 1 < Tt) tc_commit(bar(B_KEMPTY + (s + 1) % KS));
         tc_commit(bar(B_VEMPTY + s % VS));
       }
