@@ -141,6 +141,28 @@ int64_t atf_kcache_tile_keys(int d);
 atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, int64_t n, int64_t Lcap,
                            int64_t pos0, int d, void* stream);
 
+/* Decode without any device allocation.  (The paper has no counterpart: this entry point exists
+ * for the callers described here, not for a passage of the method.)
+ * Some callers can neither allocate device memory nor pass a workspace: code that runs inside
+ * another runtime's callback - a custom op of an inference server, a host that has locked its
+ * device allocator after start-up, a process held to a fixed memory budget - must not call
+ * cudaMalloc, which synchronises the device and may fail or deadlock under the host's memory
+ * manager.  atf_decode_static is atf_decode (exact mode, row-layout K cache, same arguments,
+ * same result) whose split-K scratch is a fixed array inside the library image instead of the
+ * bound workspace.  It calls no cudaMalloc, cudaFree or allocating library routine.
+ *   - Capacity: atf_decode_static_capacity() bytes (2 MiB + the 64.25 KiB header).  Every GPU
+ *     that loads the library holds that much memory until the process exits.  A problem that
+ *     needs more (roughly B*Hq*splits*(d+2)*4 bytes; e.g. B = 8, Hq = 24, d = 128 fits, B = 32
+ *     does not) is refused with ATF_ERR_WORKSPACE and a message naming both sizes.
+ *   - The first call on each device looks the array's device address up (cudaGetSymbolAddress,
+ *     with that device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each
+ *     call clears the words that must start at zero itself.  Two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it: keep calls on one device ordered. */
+size_t atf_decode_static_capacity(void);
+atf_status atf_decode_static(const void* q, const void* Kcache, const void* Vcache, void* O, int B,
+                             int Hq, int Hkv, int64_t L, int d, const int64_t* table, void* stream);
+
 /* Workspace.  The library keeps no allocation of its own: the caller allocates
  * atf_workspace_bytes() bytes of device memory (256-byte aligned), zero-fills it once, and
  * binds it (per process; the pointer is only stored).  A workspace sized for the largest call

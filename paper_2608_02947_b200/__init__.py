@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     AtfError,
     WindowTable,
     atf_decode,
+    atf_decode_static,
     atf_kcache_pack,
     atf_prefill,
     atf_rope,

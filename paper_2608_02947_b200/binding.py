@@ -57,6 +57,9 @@ def lib():
     L.atf_kcache_pack.argtypes = [vp, vp, i, i, i64, i64, i64, i, vp]
     L.atf_kcache_tile_keys.argtypes = [i]
     L.atf_kcache_tile_keys.restype = C.c_int64
+    L.atf_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
+    L.atf_decode_static.restype = C.c_int
+    L.atf_decode_static_capacity.restype = C.c_size_t
     L.atf_workspace_bytes.argtypes = [i, i, i, i, i64, i]
     L.atf_workspace_bytes.restype = C.c_size_t
     L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
@@ -246,6 +249,22 @@ def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=No
     if on_host:
         return (O.cpu(), lse.cpu()) if return_lse else O.cpu()
     return (O, lse) if return_lse else O
+
+
+def atf_decode_static(q, Kcache, Vcache, table=None, O=None):
+    """atf_decode for callers that may not allocate: the library's built-in scratch array is used
+    instead of a workspace (exact mode, row-layout cache; problems beyond its capacity raise).
+    Only argument marshalling happens here; pass O to avoid the one output allocation."""
+    for t, nm in ((q, "q"), (Kcache, "Kcache"), (Vcache, "Vcache")):
+        _dev_bf16(t, nm)
+    B, Hq, d = q.shape
+    Hkv, L = Kcache.shape[1], Kcache.shape[2]
+    if O is None:
+        O = torch.empty_like(q)
+    tab, _keep = _table_ptr(table, d)
+    _check(lib().atf_decode_static(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
+                                   C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab, _stream(q)))
+    return O
 
 
 def check_status():

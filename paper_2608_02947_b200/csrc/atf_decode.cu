@@ -17,6 +17,7 @@
 // log-sum-exp and writes O (and LSE).
 #include <algorithm>
 #include <cfloat>
+#include <cstring>
 
 #include "atf_common.cuh"
 
@@ -648,4 +649,61 @@ extern "C" atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, i
 extern "C" atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, void* O, int B, int Hq,
                                  int Hkv, int64_t L, int d, const int64_t* table, void* stream) {
   return atf_decode_ex(q, Kcache, Vcache, O, B, Hq, Hkv, L, d, table, nullptr, stream);
+}
+
+// ------------------------------------------------------------------------------------------
+// atf_decode_static: the same decode step for callers that may not allocate device memory.
+//
+// Some hosts cannot hand this library a workspace: a plug-in that runs inside another
+// runtime's callback (an inference server's custom op, a host that has locked its device
+// allocator after start-up, a process pinned to a fixed memory budget) may neither call
+// cudaMalloc - it synchronises the device and can fail or deadlock under the host's memory
+// manager - nor own a buffer of its own.  For them the split-K scratch of the decode kernel
+// (the per-split partial results and the per-(batch, KV head) split counters) lives in the
+// array below, which is part of the library image: every GPU that loads the library holds
+// these ATF_STATIC_SCRATCH_BYTES bytes until the process exits.
+//
+// In host code the array's name is only a host-side stand-in for the device object, not a
+// device address.  The address is obtained once per device, with that device current, from
+// cudaGetSymbolAddress, and that pointer is what the kernel gets.
+// ------------------------------------------------------------------------------------------
+constexpr size_t ATF_STATIC_SCRATCH_BYTES = ATF_WS_HEADER + (size_t)2 * 1024 * 1024;
+static __device__ __align__(256) unsigned char g_atf_static_scratch[ATF_STATIC_SCRATCH_BYTES];
+
+constexpr int ATF_MAX_DEVICES = 64;
+static void* g_static_scratch_ptr[ATF_MAX_DEVICES] = {nullptr};
+
+extern "C" size_t atf_decode_static_capacity(void) { return ATF_STATIC_SCRATCH_BYTES; }
+
+extern "C" atf_status atf_decode_static(const void* q, const void* Kcache, const void* Vcache, void* O, int B, int Hq,
+                                        int Hkv, int64_t L, int d, const int64_t* table, void* stream) {
+  if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || (d != 64 && d != 128) || Hq % Hkv)
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode_static: bad shape");
+  const size_t need = decode_ws_bytes(B, Hq, Hkv, L, d);
+  if (need > ATF_STATIC_SCRATCH_BYTES)
+    return atf_fail(ATF_ERR_WORKSPACE,
+                    "atf_decode_static: this problem needs %zu bytes of scratch, the built-in array holds %zu; "
+                    "use atf_decode with a bound workspace", need, ATF_STATIC_SCRATCH_BYTES);
+  int dev = -1;
+  ATF_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= ATF_MAX_DEVICES) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode_static: device index %d out of range", dev);
+  if (!g_static_scratch_ptr[dev]) {
+    // set-up, once per device, with that device current
+    void* p = nullptr;
+    ATF_CUDA_CHECK(cudaGetSymbolAddress(&p, g_atf_static_scratch));
+    if (!p) return atf_fail(ATF_ERR_CUDA, "atf_decode_static: cudaGetSymbolAddress returned a null address");
+    g_static_scratch_ptr[dev] = p;
+  }
+  void* scratch = g_static_scratch_ptr[dev];
+  // The array keeps whatever the last call left: the status words and the split counters must
+  // start at zero (a memset on the stream, not an allocation); the partials are overwritten.
+  const size_t clear = ATF_WS_STATUS_BYTES + (size_t)B * Hkv * sizeof(unsigned int);
+  ATF_CUDA_CHECK(cudaMemsetAsync(scratch, 0, clear, (cudaStream_t)stream));
+  atf_opts o;
+  memset(&o, 0, sizeof(o));
+  o.mode = ATF_MODE_EXACT;
+  o.workspace = scratch;
+  o.workspace_bytes = ATF_STATIC_SCRATCH_BYTES;
+  o.k_layout = ATF_KLAYOUT_ROWS;
+  return atf_decode_ex(q, Kcache, Vcache, O, B, Hq, Hkv, L, d, table, &o, stream);
 }
