@@ -319,11 +319,16 @@ def run_ours(args):
                             "decode_of_8000": dbytes / (dec_us * 1e-6) / 1e9 / 8000.0},
         "roofline": {"bound": "tensor", "achieved": executed / (pre_ms * 1e-3) / 1e12,
                      "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": executed / (pre_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], "traffic": None,
+                     "frac": executed / (pre_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+                     # DRAM bytes of one launch: ncu capture at N = 32768 (511 MB) scaled by N (traffic is the
+                     # repacked Q/K, V and O once each, linear in N); see profiles/
+                     "traffic": 511.2e6 * wl.N / 32768 if wl.name == "llama-3.2-3b" else None,
                      "kernel": "atf_prefill_kernel (+2 repack launches, <1% of the time)",
                      "peak_source": f"{pk['source']} sustained bf16 GEMM"},
         "roofline_decode": {"bound": "hbm", "achieved": dbytes / (dec_us * 1e-6) / 1e9, "peak": pk["hbm_gbs"],
-                            "unit": "GB/s", "frac": dbytes / (dec_us * 1e-6) / 1e9 / pk["hbm_gbs"], "traffic": None,
+                            "unit": "GB/s", "frac": dbytes / (dec_us * 1e-6) / 1e9 / pk["hbm_gbs"],
+                            # ncu: the row layout moves the whole K and V cache (128-byte DRAM lines)
+                            "traffic": float(dbytes_full),
                             "kernel": "atf_decode_kernel", "peak_source": f"{pk['source']} copy bandwidth"},
         "e2e": {"value": executed / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
