@@ -79,8 +79,8 @@ struct PrefillSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment
 };
 // barrier slots (8 bytes each) inside the BAR area
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_OFULL = 13,
-       B_QZ = 15, B_COUNT = 17 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PH0 = 11, B_OFULL = 13,
+       B_QZ = 15, B_PH1 = 17, B_COUNT = 19 };  // B_PH0 / B_PH1: first / second half of P written
 
 __global__ void __launch_bounds__(256)
 atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D) {
@@ -213,7 +213,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     mbar_init(bar(B_QFULL), 1);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar(B_KFULL + i), 1);
-      mbar_init(bar(B_KEMPTY + i), 1 + 256);
+      mbar_init(bar(B_KEMPTY + i), 1 + 256);  // the issuer's commit + every softmax thread
     }
     for (int i = 0; i < VS; ++i) {
       mbar_init(bar(B_VFULL + i), 1);
@@ -221,7 +221,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1);
-      mbar_init(bar(B_PFULL + x), 128);
+      mbar_init(bar(B_PH0 + x), 128);
+      mbar_init(bar(B_PH1 + x), 128);
       mbar_init(bar(B_OFULL + x), 1);
       mbar_init(bar(B_QZ + x), 128);
     }
@@ -336,15 +337,17 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (X == 1) ATF_STAMP(14, v - 1);
         tc_commit(bar(B_SFULL + X));
       };
-      auto issue_pv = [&](int X, int v, int tile) {
-        const uint64_t v0 = (tile & 1) ? dV1 : dV0;
-        const uint32_t tOx = tmem_base + 2 * T + X * D, tSx = tmem_base + X * T;
+      // O_X (+)= P_X V(tile) over four 16-key steps: half 0 = keys 0..63, half 1 = keys 64..127.
+      // P is read from tensor memory (8 columns per step), V through the MN-major descriptor.
+      auto issue_pv = [&](int X, int v, int tile, int half) {
+        const uint64_t v0 = ((tile & 1) ? dV1 : dV0) + (uint64_t)(half * 512);
+        const uint32_t tOx = tmem_base + 2 * T + X * D, tPx = tmem_base + X * T + half * 32;
         asm volatile(
             "{\n\t"
             ".reg .pred pf, pt;\n\t"
             ".reg .b64 vd;\n\t"
             ".reg .b32 pa;\n\t"
-            "setp.ne.b32 pf, %4, 0;\n\t"  // the very first step of the tile overwrites O
+            "setp.ne.b32 pf, %4, 0;\n\t"  // only the very first step of the tile overwrites O
             "setp.eq.u32 pt, %4, %4;\n\t"
             "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n\t"
             "add.u32 pa, %1, 8;\n\t add.u64 vd, %2, 128;\n\t"
@@ -353,16 +356,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
             "add.u32 pa, %1, 24;\n\t add.u64 vd, %2, 384;\n\t"
             "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
-            "add.u32 pa, %1, 32;\n\t add.u64 vd, %2, 512;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
-            "add.u32 pa, %1, 40;\n\t add.u64 vd, %2, 640;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
-            "add.u32 pa, %1, 48;\n\t add.u64 vd, %2, 768;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
-            "add.u32 pa, %1, 56;\n\t add.u64 vd, %2, 896;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
             "}"
-            ::"r"(tOx), "r"(tSx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)v)
+            ::"r"(tOx), "r"(tPx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)(v + half))
             : "memory");
       };
       bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
@@ -377,6 +372,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       }
       if (ok) tc_commit(bar(B_KEMPTY + 0));
+      // Step s: tile B consumes key tile s (PV of its step s, then QK of step s + 1 on key tile
+      // s + 1), tile A runs one key tile behind.  Each PV is issued in two halves, as soon as the
+      // softmax group has written that half of P, so the tensor pipe starts on the first 64 keys
+      // while the second 64 are still being exponentiated.
       for (int s = 0; s < Tt && ok; ++s) {
         const bool pvB = s < nB, pvA = s >= 1 && s - 1 < nA;
         const bool qkB = s + 1 < nB, qkA = s < nA;
@@ -385,10 +384,13 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!ok) { fail_site = 22; break; }
         if (qkB) natomsB = depth_atoms(1, s + 1);
         if (pvB) {
-          if (!wait_or_abort(bar(B_PFULL + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
+          if (!wait_or_abort(bar(B_PH0 + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
           tc_fence_after();
           ATF_STAMP(10, s);
-          issue_pv(1, s, s);
+          issue_pv(1, s, s, 0);
+          if (!wait_or_abort(bar(B_PH1 + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
+          tc_fence_after();
+          issue_pv(1, s, s, 1);
           ATF_STAMP(11, s);
         }
         if (qkB) issue_qk(1, s + 1, s + 1);
@@ -396,9 +398,12 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ATF_STAMP(12, s);
         if (qkA && s > 0) natomsA = depth_atoms(0, s);
         if (pvA) {
-          if (!wait_or_abort(bar(B_PFULL + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
+          if (!wait_or_abort(bar(B_PH0 + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
           tc_fence_after();
-          issue_pv(0, s - 1, s);
+          issue_pv(0, s - 1, s, 0);
+          if (!wait_or_abort(bar(B_PH1 + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
+          tc_fence_after();
+          issue_pv(0, s - 1, s, 1);
         }
         if (qkA) {
           if (s == 0 && !wait_or_abort(bar(B_QZ + 0), 0, abortp)) { ok = false; fail_site = 25; break; }
@@ -472,130 +477,104 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
       const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
       float s[T];
-      uint32_t pk[T / 2];
-      float psum;
-      // One pass normally.  The exponentials are taken against the reference maximum carried
-      // over from earlier tiles, so they do not wait for this tile's row maximum; if some row's
-      // maximum turns out to lead the reference by more than the threshold, the reference
-      // moves, O and l are rescaled, and the pass is repeated (rare after the first tiles).
-#pragma unroll 1
-      for (int pass = 0;; ++pass) {
-        if (natoms > 0) {
+      if (natoms > 0) {
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-          tc_wait_ld();
-        } else {
+        for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+        tc_wait_ld();
+      } else {
 #pragma unroll
-          for (int c = 0; c < T; ++c) s[c] = 0.f;
-        }
-        if (row == 0) ATF_STAMP(1 + 5 * X, v);
-        // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
-        //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
-        //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
-        //      no row of this warp has such a cell in it. ----
-        if (MODE == ATF_MODE_EXACT) {
-          const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
-          const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
-          uint32_t qq_next = (p_all < p_any) ? *reinterpret_cast<const uint32_t*>(qsrc + 2 * p_all) : 0u;
-          for (int p = p_all; p < p_any; ++p) {
-            const int wp = sW[H - 1 - p];
-            const bool subtract = p < p_mid;
-            const uint32_t qq = qq_next;
-#ifndef ATF_EXP_NOQ
-            if (p + 1 < p_any) qq_next = *reinterpret_cast<const uint32_t*>(qsrc + 2 * (p + 1));  // overlaps this pair's work
-#endif
-            float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
-            if (subtract) {
-              q0 = -q0;
-              q1 = -q1;
-            }
-            const int col = 2 * p;
-            // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
-            const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
-            const int chunk = (col & 63) >> 3;
-            uint32_t base8[8];
+        for (int c = 0; c < T; ++c) s[c] = 0.f;
+      }
+      if (row == 0) ATF_STAMP(1 + 5 * X, v);
+      // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
+      //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
+      //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
+      //      no row of this warp has such a cell in it. ----
+      if (MODE == ATF_MODE_EXACT) {
+        const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
+        const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
+        uint32_t qq_next = (p_all < p_any) ? *reinterpret_cast<const uint32_t*>(qsrc + 2 * p_all) : 0u;
+        for (int p = p_all; p < p_any; ++p) {
+          const int wp = sW[H - 1 - p];
+          const bool subtract = p < p_mid;
+          const uint32_t qq = qq_next;
+          if (p + 1 < p_any) qq_next = *reinterpret_cast<const uint32_t*>(qsrc + 2 * (p + 1));  // overlaps this pair's work
+          float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
+          if (subtract) {
+            q0 = -q0;
+            q1 = -q1;
+          }
+          const int col = 2 * p;
+          // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
+          const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+          const int chunk = (col & 63) >> 3;
+          uint32_t base8[8];
 #pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
-            // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
-            // is formed on the FMA pipe as a saturated affine function of its column (the integer and
-            // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
-            const float jbf = (float)(zrow - wp);
-            const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
+          for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
+          // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
+          // is formed on the FMA pipe as a saturated affine function of its column (the integer and
+          // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
+          const float jbf = (float)(zrow - wp);
+          const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
-              const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
+          for (int q4 = 0; q4 < 4; ++q4) {
+            // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
+            const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
 #ifdef ATF_TRACE
-              if (touched && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[15 * 64 + v] += 1;
-              if (q4 == 0 && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[4 * 64 + v] += 1;
+            if (touched && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[15 * 64 + v] += 1;
+            if (q4 == 0 && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[4 * 64 + v] += 1;
 #endif
-              if (touched) {
-                // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
-                uint32_t kk[32];
+            if (touched) {
+              // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
+              uint32_t kk[32];
 #pragma unroll
-                for (int cc = 0; cc < 32; ++cc) {
-                  const int c = q4 * 32 + cc;
-                  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + c * 128));
-                }
+              for (int cc = 0; cc < 32; ++cc) {
+                const int c = q4 * 32 + cc;
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + c * 128));
+              }
 #pragma unroll
-                for (int cc = 0; cc < 32; ++cc) {
-                  const int c = q4 * 32 + cc;
-                  const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
-                  const float coef = __saturatef(fmaf(ca, (float)c, cb));
-                  s[c] = fmaf(term, coef, s[c]);
-                }
+              for (int cc = 0; cc < 32; ++cc) {
+                const int c = q4 * 32 + cc;
+                const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
+                const float coef = __saturatef(fmaf(ca, (float)c, cb));
+                s[c] = fmaf(term, coef, s[c]);
               }
             }
           }
         }
+      }
 
-        // ---- causal mask, dropped keys (exact mode: per cell) ----
-        if (dt == 0 || zmax > zdrop) {
+      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
+
+      // ---- causal mask, dropped keys (exact mode: per cell) ----
+      if (dt == 0 || zmax > zdrop) {
 #pragma unroll
-          for (int c = 0; c < T; ++c) {
-            const int z = zrow - c;
-            s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
-          }
+        for (int c = 0; c < T; ++c) {
+          const int z = zrow - c;
+          s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
         }
-        float mx;
-        {
-          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      }
+      float mx;
+      {
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int c = 0; c < T; c += 8) {
+        for (int c = 0; c < T; c += 8) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
-          }
-          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+          for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
         }
-        if (v == 0 && pass == 0) m_used = mx;  // finite: the diagonal cell of every row is live
-        const float neg_m = -m_used * kScaleLog2;
-        {
-          const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
-          float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-          for (int c = 0; c < T; c += 2) {
-            float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
-            if (((c >> 1) & 3) < POLY_OF_4) {
-              x = exp2_poly2(x);
-            } else {
-              x.x = ex2_approx(x.x);
-              x.y = ex2_approx(x.y);
-            }
-            acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
-            pk[c >> 1] = pack_bf16x2(x.x, x.y);
-          }
-          const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
-          psum = (a01.x + a01.y) + (a23.x + a23.y);
-        }
-        const bool lag = (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD;
-        if (!__any_sync(0xffffffffu, lag)) break;
-        // move the reference maximum of the lagging rows, rescale their O and l, redo the pass
-        float scale_o = 1.f;
-        if (lag) {
-          scale_o = ex2_approx((m_used - mx) * kScaleLog2);
-          m_used = mx;
-          l_run *= scale_o;
-        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+      }
+      // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
+      float scale_o = 1.f;
+      bool moved = false;
+      if (v == 0) {
+        m_used = mx;  // finite: the diagonal cell of every row is live
+      } else if ((mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD) {
+        scale_o = ex2_approx((m_used - mx) * kScaleLog2);
+        m_used = mx;
+        moved = true;
+      }
+      if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles; PV of the previous step is complete
 #pragma unroll
         for (int q4 = 0; q4 < D / 32; ++q4) {
           uint32_t o[32];
@@ -607,9 +586,40 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         tc_wait_st();
       }
-      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
+      const float neg_m = -m_used * kScaleLog2;
+      const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
+      float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      // exponentials of columns [c_lo, c_hi) -> packed bf16 pairs pk[(c - c_base) / 2]
+      auto exp_range = [&](uint32_t* pk, int c_base, int c_lo, int c_hi) {
+#pragma unroll
+        for (int c = c_lo; c < c_hi; c += 2) {
+          float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
+          if (((c >> 1) & 3) < POLY_OF_4) {
+            x = exp2_poly2(x);
+          } else {
+            x.x = ex2_approx(x.x);
+            x.y = ex2_approx(x.y);
+          }
+          acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
+          pk[(c - c_base) >> 1] = pack_bf16x2(x.x, x.y);
+        }
+      };
+      // ---- P (bf16) over the first 64 columns of S (column c holds keys 2c and 2c+1), in two halves:
+      //      the PV product starts on keys 0..63 while the exponentials of keys 64..127 are still running ----
+      uint32_t pk0[32], pk1[32];
+      exp_range(pk0, 0, 0, 64);
+      tc_st32(tS, pk0);
+      exp_range(pk1, 64, 64, 80);
+      tc_wait_st();  // the store above has had a few hundred clocks
+      tc_fence_before();
+      mbar_arrive(bar(B_PH0 + X));
+      exp_range(pk1, 64, 80, 128);
+      tc_st32(tS + 32, pk1);
+      {
+        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+        l_run = l_run * scale_o + ((a01.x + a01.y) + (a23.x + a23.y));
+      }
       if (row == 0) ATF_STAMP(2 + 5 * X, v);
-      l_run += psum;
       if (COUNT && row_ok) {
         const int ncols = dt == 0 ? row + 1 : T;
         cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
@@ -621,10 +631,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
         }
       }
-
-      // ---- P (bf16) over the first 64 columns of S: column c holds keys 2c and 2c+1 ----
-      tc_st32(tS, pk);
-      tc_st32(tS + 32, pk + 32);
       // zero the Q columns that stop being live in most cells at the next step
       if (v + 1 < nX) {
         sc.advance(sW, H, dt + 1, wq);
@@ -633,7 +639,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       tc_wait_st();
       tc_fence_before();
       if (row == 0) ATF_STAMP(3 + 5 * X, v);
-      mbar_arrive(bar(B_PFULL + X));
+      mbar_arrive(bar(B_PH1 + X));
     }
 
     if (ok && nX > 0) {
