@@ -12,12 +12,16 @@
 // B (the next 128), and walks the key tiles from B's diagonal outwards.  Warp roles:
 //   warp 0      TMA producer: Q once, then K (live 64-column blocks only) and V tiles into
 //               two-stage rings of 128-byte-swizzled shared memory;
-//   warp 1      MMA issuer (one thread): S_X = Q_X K^T over the live depth into tensor memory,
-//               O_X += P_X V with P read from tensor memory; the two query tiles alternate
-//               so that the tensor pipe works on one while the other is in its softmax;
+//   warps 1, 2  MMA issuers (one thread each) of tile B and tile A: S_X = Q_X K^T over the live
+//               depth into tensor memory, O_X += P_X V with P read from tensor memory;
 //   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one query row per thread:
 //               read S, finish the window rule, mask, online softmax with lazy rescaling of
 //               O, write P (bf16) over S in tensor memory.
+// A key tile is processed as two halves of 64 keys.  Each half of a query tile's 128 S columns
+// is a buffer of its own: when the softmax group has turned S(v, h) into P(v, h) the issuer
+// runs O += P(v, h) V(half h) and then S(v + 1, h) into the same columns, while the group is
+// already working on the other half.  The softmax groups, which are the busiest unit of the
+// kernel (one MUFU exponential per cell), so never wait for a product that is not yet issued.
 //
 // Exact mode (the per-term definition).  For a tile at tile distance D the cells span
 // distances [z_min, z_max].  Pairs with w >= z_max are live in every cell: they are the MMA
@@ -38,6 +42,9 @@ constexpr int T = 128;              // query rows per tile and key columns per t
 constexpr int BLK_BYTES = T * 128;  // one [128 x 64] bf16 block, 128-byte rows
 constexpr int KS = 2, VS = 2;       // ring depths
 constexpr int PF_THREADS = 384;
+#ifndef ATF_PRODUCER_WARP
+#define ATF_PRODUCER_WARP 0
+#endif
 // Register budget.  The kernel is compiled for 168 registers per thread (65536 / 384, rounded
 // down to a multiple of 8), i.e. 64512 in use at launch.  The producer/MMA warpgroup then
 // shrinks to 72 and the two softmax warpgroups grow to 216: 128*72 + 256*216 = 64512.  The
@@ -79,8 +86,10 @@ struct PrefillSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment
 };
 // barrier slots (8 bytes each) inside the BAR area
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PH0 = 11, B_OFULL = 13,
-       B_QZ = 15, B_PH1 = 17, B_COUNT = 19 };  // B_PH0 / B_PH1: first / second half of P written
+// B_SFULL / B_PFULL: slot + 2 * X + h for query tile X (0 = A, 1 = B) and key half h of the tile
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 13, B_OFULL = 17,
+       B_QZ = 19, B_COUNT = 21 };
+constexpr int HK = T / 2;  // keys per half tile: S and P are produced and consumed in halves
 
 __global__ void __launch_bounds__(256)
 atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D) {
@@ -136,7 +145,7 @@ __device__ __forceinline__ int tile_depth(int H, int p_any, int p_mid, int dt) {
 // of 2^f on f = x - n in [-0.5, 0.5] (relative error < 8e-5, below the bf16 rounding of P),
 // and add n to the exponent field.
 #ifndef ATF_POLY_OF_4
-#define ATF_POLY_OF_4 0
+#define ATF_POLY_OF_4 1
 #endif
 constexpr int POLY_OF_4 = ATF_POLY_OF_4;  // of every 4 packed pairs, this many take the polynomial, the rest MUFU
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
@@ -185,7 +194,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   constexpr int H = D / 2;
   constexpr int NB = D / 64;
   constexpr uint32_t TMEM_COLS = 512;
-  constexpr uint32_t IDESC_QK = make_idesc_bf16(128, T, 0, 0);
+  constexpr uint32_t IDESC_QK = make_idesc_bf16(128, HK, 0, 0);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(128, D, 0, 1);
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
 
@@ -198,6 +207,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + SM::BAR_OFF + 8 * B_COUNT);
   __shared__ int sW[ATF_MAX_PAIRS];
   __shared__ int s_abort;
+  __shared__ int s_nat[2][2];  // MMA depth of query tile X at its next step (by step parity), from its softmax group
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int npt = (P.N + 2 * T - 1) / (2 * T);
@@ -213,16 +223,17 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     mbar_init(bar(B_QFULL), 1);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar(B_KFULL + i), 1);
-      mbar_init(bar(B_KEMPTY + i), 1 + 256);  // the issuer's commit + every softmax thread
+      mbar_init(bar(B_KEMPTY + i), 256);  // every softmax thread, once it has seen both halves of S of its tile
     }
     for (int i = 0; i < VS; ++i) {
       mbar_init(bar(B_VFULL + i), 1);
-      mbar_init(bar(B_VEMPTY + i), 1);
+      mbar_init(bar(B_VEMPTY + i), 2);  // one arrival per MMA issuer
     }
     for (int x = 0; x < 2; ++x) {
-      mbar_init(bar(B_SFULL + x), 1);
-      mbar_init(bar(B_PH0 + x), 128);
-      mbar_init(bar(B_PH1 + x), 128);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(bar(B_SFULL + 2 * x + h), 1);
+        mbar_init(bar(B_PFULL + 2 * x + h), 128);
+      }
       mbar_init(bar(B_OFULL + x), 1);
       mbar_init(bar(B_QZ + x), 128);
     }
@@ -249,7 +260,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   volatile int* abortp = &s_abort;
   unsigned int fail_site = 0;
 
-  if (warp == 0) {
+  if (warp == ATF_PRODUCER_WARP) {
     // =============================== TMA producer ===============================
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
@@ -276,33 +287,29 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tma_load_3d(sV + vs * SM::TILE + kb * BLK_BYTES, &tmV, bar(B_VFULL + vs), kb * 64, j * T, bhk);
       }
     }
-  } else if (warp == 1) {
-    // =============================== MMA issuer ===============================
+  } else if (warp == 1 || warp == 2) {
+    // =============================== MMA issuers ===============================
+    // warp 1 serves query tile B, warp 2 query tile A (one thread each).  A tcgen05.mma issue
+    // blocks while the tensor pipe's queue is full and a lone thread runs its bookkeeping slowly,
+    // so two issuers keep the pipe fed where one could not.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
       static_assert(KS == 2 && VS == 2, "stage selection below assumes two-stage rings");
-      TileSched scA, scB;
+      const int X = warp == 1 ? 1 : 0;
+      const int nX = X ? nB : nA;
+      const int toff = X ? 0 : 1;  // step v of this query tile works on key tile v + toff
       // Descriptors are built once; an MMA step only adds a constant to the start-address field
       // (16-byte units): K-major operands advance 32 bytes per 16-column step inside a
       // 64-column block and one block per four steps; V advances 16 key rows (2048 bytes).
-      const uint64_t dQ0 = make_smem_desc_sw128(sQ, 16, 1024), dQ1 = make_smem_desc_sw128(sQ + SM::TILE, 16, 1024);
+      const uint64_t dQ = make_smem_desc_sw128(sQ + X * SM::TILE, 16, 1024);
       const uint64_t dK0 = make_smem_desc_sw128(sK, 16, 1024), dK1 = make_smem_desc_sw128(sK + SM::TILE, 16, 1024);
       const uint64_t dV0 = make_smem_desc_sw128(sV, BLK_BYTES, 1024),
                      dV1 = make_smem_desc_sw128(sV + SM::TILE, BLK_BYTES, 1024);
-      // S_X = Q_X K(tile)^T for step v of tile X (X: 0 = A, 1 = B)
-      // live depth (in 16-column MMA steps) of step v of tile X; computed ahead of time, while the
-      // issuer would otherwise be waiting, because a lone thread runs such code slowly
-      auto depth_atoms = [&](int X, int v) {
-        TileSched& sc = X ? scB : scA;
-        sc.advance(sW, H, v, 0);
-        return (tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, v) + 7) / 8;
-      };
-      int natomsA = depth_atoms(0, 0), natomsB = depth_atoms(1, 0);
-      auto issue_qk = [&](int X, int v, int tile) {
-        const int natoms = X ? natomsB : natomsA;
-        const uint64_t dQ = X ? dQ1 : dQ0, k0 = (tile & 1) ? dK1 : dK0;
-        const uint32_t tSx = tmem_base + X * T;
-        if (X == 1) ATF_STAMP(13, v - 1);
+      // S_X(half h) = Q_X K(tile, keys 64h..64h+63)^T over natoms 16-column steps, into columns
+      // [64h, 64h+64) of the tile's S region; then signal the softmax group.
+      auto issue_qk = [&](int tile, int h, int natoms) {
+        const uint64_t k0 = ((tile & 1) ? dK1 : dK0) + (uint64_t)(h * 512);
+        const uint32_t tSx = tmem_base + X * T + h * HK;
         asm volatile(
             "{\n\t"
             ".reg .pred pf, p0, p1, p2, p3, p4, p5, p6, p7;\n\t"
@@ -334,20 +341,19 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             "}"
             ::"r"(tSx), "l"(dQ), "l"(k0), "r"(IDESC_QK), "r"((uint32_t)natoms)
             : "memory");
-        if (X == 1) ATF_STAMP(14, v - 1);
-        tc_commit(bar(B_SFULL + X));
       };
-      // O_X (+)= P_X V(tile) over four 16-key steps: half 0 = keys 0..63, half 1 = keys 64..127.
-      // P is read from tensor memory (8 columns per step), V through the MN-major descriptor.
-      auto issue_pv = [&](int X, int v, int tile, int half) {
-        const uint64_t v0 = ((tile & 1) ? dV1 : dV0) + (uint64_t)(half * 512);
-        const uint32_t tOx = tmem_base + 2 * T + X * D, tPx = tmem_base + X * T + half * 32;
+      // O_X (+)= P_X(half h) V(tile, keys 64h..64h+63) over four 16-key steps.  P is read from
+      // tensor memory (8 columns per step, at the start of the half's S columns), V through the
+      // MN-major descriptor.  `first` marks the very first product of the query tile.
+      auto issue_pv = [&](int tile, int h, bool first) {
+        const uint64_t v0 = ((tile & 1) ? dV1 : dV0) + (uint64_t)(h * 512);
+        const uint32_t tOx = tmem_base + 2 * T + X * D, tPx = tmem_base + X * T + h * HK;
         asm volatile(
             "{\n\t"
             ".reg .pred pf, pt;\n\t"
             ".reg .b64 vd;\n\t"
             ".reg .b32 pa;\n\t"
-            "setp.ne.b32 pf, %4, 0;\n\t"  // only the very first step of the tile overwrites O
+            "setp.eq.b32 pf, %4, 0;\n\t"  // only the very first step of the tile overwrites O
             "setp.eq.u32 pt, %4, %4;\n\t"
             "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n\t"
             "add.u32 pa, %1, 8;\n\t add.u64 vd, %2, 128;\n\t"
@@ -357,64 +363,66 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             "add.u32 pa, %1, 24;\n\t add.u64 vd, %2, 384;\n\t"
             "tcgen05.mma.cta_group::1.kind::f16 [%0], [pa], vd, %3, pt;\n\t"
             "}"
-            ::"r"(tOx), "r"(tPx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)(v + half))
+            ::"r"(tOx), "r"(tPx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)(first ? 1 : 0))
             : "memory");
       };
-      bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
+      // Each half of a query tile's S region is its own buffer: as soon as the softmax group has
+      // turned S(v, h) into P(v, h), the issuer runs O += P(v, h) V and then S(v + 1, h) into the
+      // same columns (the tensor pipe executes one thread's products in issue order), while the
+      // group is already working on the other half.  The softmax groups therefore never wait
+      // for the tensor pipe as long as it keeps up.
+      // A V stage is released by one arrival per issuer; an issuer that has no use for a key
+      // tile still accounts for it, once the tile has been loaded (so that the arrival falls
+      // into the right phase of the barrier).
+      auto skip_v = [&](int t) {
+        if (!wait_or_abort(bar(B_VFULL + t % VS), (t / VS) & 1, abortp)) return false;
+        mbar_arrive(bar(B_VEMPTY + t % VS));
+        return true;
+      };
+      bool ok = wait_or_abort(bar(B_QFULL), 0, abortp) && wait_or_abort(bar(B_QZ + X), 0, abortp);
       if (!ok) fail_site = 20;
-      if (ok && nB > 0) {
-        ok = wait_or_abort(bar(B_KFULL + 0), 0, abortp) && wait_or_abort(bar(B_QZ + 1), 0, abortp);
+      for (int t = 0; t < toff && ok; ++t) ok = skip_v(t);
+      int natoms = 0;
+      if (ok && nX > 0) {
+        TileSched sc0;
+        sc0.advance(sW, H, 0, 0);
+        natoms = (tile_depth<MODE>(H, H - sc0.r_any, H - sc0.r_mid, 0) + 7) / 8;
+        ok = wait_or_abort(bar(B_KFULL + toff % KS), (toff / KS) & 1, abortp);
         if (ok) {
           tc_fence_after();
-          issue_qk(1, 0, 0);
+          issue_qk(toff, 0, natoms);
+          tc_commit(bar(B_SFULL + 2 * X));
+          issue_qk(toff, 1, natoms);
+          tc_commit(bar(B_SFULL + 2 * X + 1));
         } else {
           fail_site = 21;
         }
       }
-      if (ok) tc_commit(bar(B_KEMPTY + 0));
-      // Step s: tile B consumes key tile s (PV of its step s, then QK of step s + 1 on key tile
-      // s + 1), tile A runs one key tile behind.  Each PV is issued in two halves, as soon as the
-      // softmax group has written that half of P, so the tensor pipe starts on the first 64 keys
-      // while the second 64 are still being exponentiated.
-      for (int s = 0; s < Tt && ok; ++s) {
-        const bool pvB = s < nB, pvA = s >= 1 && s - 1 < nA;
-        const bool qkB = s + 1 < nB, qkA = s < nA;
-        if (pvB || pvA) ok = ok && wait_or_abort(bar(B_VFULL + s % VS), (s / VS) & 1, abortp);
-        if (qkB || qkA) ok = ok && wait_or_abort(bar(B_KFULL + (s + 1) % KS), ((s + 1) / KS) & 1, abortp);
+      for (int v = 0; v < nX && ok; ++v) {
+        const int t = v + toff;
+        const bool more = v + 1 < nX;
+        ok = wait_or_abort(bar(B_VFULL + t % VS), (t / VS) & 1, abortp);
+        if (more) ok = ok && wait_or_abort(bar(B_KFULL + (t + 1) % KS), ((t + 1) / KS) & 1, abortp);
         if (!ok) { fail_site = 22; break; }
-        if (qkB) natomsB = depth_atoms(1, s + 1);
-        if (pvB) {
-          if (!wait_or_abort(bar(B_PH0 + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (!wait_or_abort(bar(B_PFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 23; break; }
           tc_fence_after();
-          ATF_STAMP(10, s);
-          issue_pv(1, s, s, 0);
-          if (!wait_or_abort(bar(B_PH1 + 1), s & 1, abortp)) { ok = false; fail_site = 23; break; }
-          tc_fence_after();
-          issue_pv(1, s, s, 1);
-          ATF_STAMP(11, s);
+          if (h == 0 && more) natoms = *reinterpret_cast<volatile int*>(&s_nat[X][(v + 1) & 1]);
+          if (X == 1) ATF_STAMP(10, 2 * v + h);
+          issue_pv(t, h, v == 0 && h == 0);
+          if (X == 1) ATF_STAMP(11, 2 * v + h);
+          if (more) issue_qk(t + 1, h, natoms);
+          if (X == 1) ATF_STAMP(12, 2 * v + h);
+          tc_commit(bar(B_SFULL + 2 * X + h));  // S(v + 1, h) is there, and every product before it is complete
+          if (X == 1) ATF_STAMP(13, 2 * v + h);
         }
-        if (qkB) issue_qk(1, s + 1, s + 1);
-        else if (pvB) tc_commit(bar(B_OFULL + 1));
-        ATF_STAMP(12, s);
-        if (qkA && s > 0) natomsA = depth_atoms(0, s);
-        if (pvA) {
-          if (!wait_or_abort(bar(B_PH0 + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
-          tc_fence_after();
-          issue_pv(0, s - 1, s, 0);
-          if (!wait_or_abort(bar(B_PH1 + 0), (s - 1) & 1, abortp)) { ok = false; fail_site = 24; break; }
-          tc_fence_after();
-          issue_pv(0, s - 1, s, 1);
-        }
-        if (qkA) {
-          if (s == 0 && !wait_or_abort(bar(B_QZ + 0), 0, abortp)) { ok = false; fail_site = 25; break; }
-          tc_fence_after();
-          issue_qk(0, s, s + 1);
-        } else if (pvA) {
-          tc_commit(bar(B_OFULL + 0));
-        }
-        if (s + 1 < Tt) tc_commit(bar(B_KEMPTY + (s + 1) % KS));
-        tc_commit(bar(B_VEMPTY + s % VS));
+        if (!ok) break;
+        if (!more) tc_commit(bar(B_OFULL + X));
+        tc_commit(bar(B_VEMPTY + t % VS));
       }
+      for (int t = toff + nX; t < Tt && ok; ++t) ok = skip_v(t);
+      if (!ok && !fail_site) fail_site = 25;
     }
   } else if (warp >= 4) {
     // =============================== softmax groups ===============================
@@ -453,8 +461,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_arrive(bar(B_QZ + X));
     }
 
-    float m_used = -INFINITY, l_run = 0.f;  // m_used in raw score units
+    float m_used = -INFINITY, l_run = 0.f;  // m_used in raw score units; -inf until a live cell is seen
     unsigned long long cnt = 0;
+    const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
+    const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
 
     for (int t = 0; t < Tt && ok; ++t) {
       const int v = X ? t : t - 1;  // step of this query tile = its tile distance to key tile t
@@ -470,178 +480,205 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int p_any = H - sc.r_any, p_mid = H - sc.r_mid, p_all = H - sc.r_all;  // cursors already at dt
       const int depth = tile_depth<MODE>(H, p_any, p_mid, dt);
       const int natoms = (depth + 7) / 8;
-      if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
-      tc_fence_after();
-      if (row == 0) ATF_STAMP(0 + 5 * X, v);
-
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
-      const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
-      float s[T];
-      if (natoms > 0) {
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-        tc_wait_ld();
-      } else {
-#pragma unroll
-        for (int c = 0; c < T; ++c) s[c] = 0.f;
-      }
-      if (row == 0) ATF_STAMP(1 + 5 * X, v);
-      // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
-      //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
-      //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
-      //      no row of this warp has such a cell in it. ----
-      if (MODE == ATF_MODE_EXACT) {
-        const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // distances to column 0 over the warp
-        const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
-        uint32_t qq_next = (p_all < p_any) ? *reinterpret_cast<const uint32_t*>(qsrc + 2 * p_all) : 0u;
-        for (int p = p_all; p < p_any; ++p) {
-          const int wp = sW[H - 1 - p];
-          const bool subtract = p < p_mid;
-          const uint32_t qq = qq_next;
-          if (p + 1 < p_any) qq_next = *reinterpret_cast<const uint32_t*>(qsrc + 2 * (p + 1));  // overlaps this pair's work
-          float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
-          if (subtract) {
-            q0 = -q0;
-            q1 = -q1;
-          }
-          const int col = 2 * p;
-          // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
-          const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
-          const int chunk = (col & 63) >> 3;
-          uint32_t base8[8];
-#pragma unroll
-          for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
-          // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
-          // is formed on the FMA pipe as a saturated affine function of its column (the integer and
-          // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
-          const float jbf = (float)(zrow - wp);
-          const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            // distances of the warp's cells in this chunk span [zw_lo - 32*q4 - 31, zw_hi - 32*q4]
-            const bool touched = subtract ? (zw_hi - 32 * q4 > wp) : (zw_lo - 32 * q4 - 31 <= wp && zw_hi - 32 * q4 >= 0);
+      const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // the same over the warp's rows
+
+#pragma unroll 1
+      for (int h = 0; h < 2; ++h) {
+        const int c0 = h * HK;  // first key column of this half
+        if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 32; break; }
+        tc_fence_after();
+        if (row == 0) ATF_STAMP(0 + 5 * X, 2 * v + h);
 #ifdef ATF_TRACE
-            if (touched && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[15 * 64 + v] += 1;
-            if (q4 == 0 && row == 0 && X == 1 && blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && v < 64) P.trace[4 * 64 + v] += 1;
+        const bool tr1 = X == 1 && lane == 0 && (warp & 3) == 1;
+        if (tr1) ATF_STAMP(4, 2 * v + h);
 #endif
-            if (touched) {
-              // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
-              uint32_t kk[32];
+        float s[HK];
+        if (natoms > 0) {
+          tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
+          tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
+          tc_wait_ld();
+        } else {
 #pragma unroll
-              for (int cc = 0; cc < 32; ++cc) {
-                const int c = q4 * 32 + cc;
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + c * 128));
-              }
+          for (int c = 0; c < HK; ++c) s[c] = 0.f;
+        }
+        
+#ifdef ATF_TRACE
+        if (tr1) ATF_STAMP(6, 2 * v + h);
+#endif
+        // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
+        //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
+        //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
+        //      no row of this warp has such a cell in it. ----
+        if (MODE == ATF_MODE_EXACT) {
+          for (int p = p_all; p < p_any; ++p) {
+            const int wp = sW[H - 1 - p];
+            const bool subtract = p < p_mid;
+            // distances of the warp's cells in chunk q (columns c0 + 32q ..) span
+            // [zw_lo - c0 - 32q - 31, zw_hi - c0 - 32q]
+            bool touched[2];
 #pragma unroll
-              for (int cc = 0; cc < 32; ++cc) {
-                const int c = q4 * 32 + cc;
-                const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
-                const float coef = __saturatef(fmaf(ca, (float)c, cb));
-                s[c] = fmaf(term, coef, s[c]);
+            for (int q = 0; q < 2; ++q) {
+              const int hi = zw_hi - c0 - 32 * q, lo = zw_lo - c0 - 32 * q - 31;
+              touched[q] = subtract ? (hi > wp) : (lo <= wp && hi >= 0);
+            }
+            if (!touched[0] && !touched[1]) continue;
+            const uint32_t qq = *reinterpret_cast<const uint32_t*>(qsrc + 2 * p);
+            float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
+            if (subtract) {
+              q0 = -q0;
+              q1 = -q1;
+            }
+            const int col = 2 * p;
+            // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
+            const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+            const int chunk = (col & 63) >> 3;
+            uint32_t base8[8];
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
+            // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
+            // is formed on the FMA pipe as a saturated affine function of its column (the integer and
+            // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
+            const float jbf = (float)(zrow - wp - c0);
+            const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              if (touched[q]) {
+                // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
+                uint32_t kk[32];
+#pragma unroll
+                for (int cc = 0; cc < 32; ++cc) {
+                  const int c = q * 32 + cc;
+                  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + (c0 + c) * 128));
+                }
+#pragma unroll
+                for (int cc = 0; cc < 32; ++cc) {
+                  const int c = q * 32 + cc;
+                  const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
+                  const float coef = __saturatef(fmaf(ca, (float)c, cb));
+                  s[c] = fmaf(term, coef, s[c]);
+                }
               }
             }
           }
         }
-      }
+        if (h == 1) mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
 
-      mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
-
-      // ---- causal mask, dropped keys (exact mode: per cell) ----
-      if (dt == 0 || zmax > zdrop) {
+#ifdef ATF_TRACE
+        if (tr1) ATF_STAMP(14, 2 * v + h);
+#endif
+        // ---- causal mask, dropped keys (exact mode: per cell) ----
+        if (dt == 0 || zmax > zdrop) {
 #pragma unroll
-        for (int c = 0; c < T; ++c) {
-          const int z = zrow - c;
-          s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
+          for (int c = 0; c < HK; ++c) {
+            const int z = zrow - c0 - c;
+            s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
+          }
         }
-      }
-      float mx;
-      {
-        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        float mx;
+        {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < T; c += 8) {
+          for (int c = 0; c < HK; c += 8) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+            for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+          }
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+#ifdef ATF_X_NOMAX
+          mx = s[0] + s[63];
+#endif
         }
-        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-      }
-      // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
-      float scale_o = 1.f;
-      bool moved = false;
-      if (v == 0) {
-        m_used = mx;  // finite: the diagonal cell of every row is live
-      } else if ((mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD) {
-        scale_o = ex2_approx((m_used - mx) * kScaleLog2);
-        m_used = mx;
-        moved = true;
-      }
-      if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles; PV of the previous step is complete
-#pragma unroll
-        for (int q4 = 0; q4 < D / 32; ++q4) {
-          uint32_t o[32];
-          tc_ld32(tO + q4 * 32, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
-          tc_st32(tO + q4 * 32, o);
+        // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
+        // (or when the row sees its first live cell)
+        float scale_o = 1.f;
+        bool moved = false;
+        if (mx > m_used && (m_used == -INFINITY || (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD)) {
+          scale_o = m_used == -INFINITY ? 0.f : ex2_approx((m_used - mx) * kScaleLog2);
+          m_used = mx;
+          moved = !(v == 0 && h == 0);  // nothing has been accumulated before the first half
         }
-        tc_wait_st();
-      }
-      const float neg_m = -m_used * kScaleLog2;
-      const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
-      float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-      // exponentials of columns [c_lo, c_hi) -> packed bf16 pairs pk[(c - c_base) / 2]
-      auto exp_range = [&](uint32_t* pk, int c_base, int c_lo, int c_hi) {
+        if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles
+          // every product issued so far must be complete: the issuer signals the other half's S
+          // barrier after each product (S(v, 1) follows P(v-1, 1) V; S(v+1, 0) follows P(v, 0) V)
+          const int vo = h == 0 ? v : v + 1;
+          if (!wait_or_abort(bar(B_SFULL + 2 * X + (h ^ 1)), vo & 1, abortp)) { ok = false; fail_site = 34; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int c = c_lo; c < c_hi; c += 2) {
+          for (int q4 = 0; q4 < D / 32; ++q4) {
+            uint32_t o[32];
+            tc_ld32(tO + q4 * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
+            tc_st32(tO + q4 * 32, o);
+          }
+          tc_wait_st();
+        }
+#ifdef ATF_TRACE
+        if (tr1) ATF_STAMP(7, 2 * v + h);
+#endif
+        const float neg_m = m_used == -INFINITY ? 0.f : -m_used * kScaleLog2;
+        const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
+        float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        // ---- P (bf16) over the first 32 columns of this half of S (column c holds keys 2c and 2c+1) ----
+        uint32_t pk[HK / 2];
+#pragma unroll
+        for (int c = 0; c < HK; c += 2) {
           float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
           if (((c >> 1) & 3) < POLY_OF_4) {
             x = exp2_poly2(x);
           } else {
+#ifndef ATF_X_NOEXP
             x.x = ex2_approx(x.x);
             x.y = ex2_approx(x.y);
+#endif
           }
           acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
-          pk[(c - c_base) >> 1] = pack_bf16x2(x.x, x.y);
+          pk[c >> 1] = pack_bf16x2(x.x, x.y);
         }
-      };
-      // ---- P (bf16) over the first 64 columns of S (column c holds keys 2c and 2c+1), in two halves:
-      //      the PV product starts on keys 0..63 while the exponentials of keys 64..127 are still running ----
-      uint32_t pk0[32], pk1[32];
-      exp_range(pk0, 0, 0, 64);
-      tc_st32(tS, pk0);
-      exp_range(pk1, 64, 64, 80);
-      tc_wait_st();  // the store above has had a few hundred clocks
-      tc_fence_before();
-      mbar_arrive(bar(B_PH0 + X));
-      exp_range(pk1, 64, 80, 128);
-      tc_st32(tS + 32, pk1);
-      {
-        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
-        l_run = l_run * scale_o + ((a01.x + a01.y) + (a23.x + a23.y));
-      }
-      if (row == 0) ATF_STAMP(2 + 5 * X, v);
-      if (COUNT && row_ok) {
-        const int ncols = dt == 0 ? row + 1 : T;
-        cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
-        if (MODE == ATF_MODE_EXACT) {
-          for (int p = p_all; p < p_any; ++p) {
-            const int wp = sW[H - 1 - p];
-            const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
-            cnt += (unsigned long long)max(0, hi - lo + 1);
+        tc_st32(tS + c0, pk);
+#ifdef ATF_TRACE
+        if (tr1) ATF_STAMP(9, 2 * v + h);
+#endif
+        {
+          const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+          l_run = l_run * scale_o + ((a01.x + a01.y) + (a23.x + a23.y));
+        }
+        
+        if (h == 0) {
+          if (COUNT && row_ok) {
+            const int ncols = dt == 0 ? row + 1 : T;
+            cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
+            if (MODE == ATF_MODE_EXACT) {
+              for (int p = p_all; p < p_any; ++p) {
+                const int wp = sW[H - 1 - p];
+                const int lo = max(0, zrow - wp), hi = min(T - 1, zrow);
+                cnt += (unsigned long long)max(0, hi - lo + 1);
+              }
+            }
+          }
+          // Zero the Q columns that stop being live in most cells at the next step.  S(v + 1, 0) is
+          // issued once this half of P is signalled, so the zeroing has to happen here; S(v, 1) still
+          // needs the columns, so wait until it has been computed (it was issued long ago).
+          if (v + 1 < nX) {
+            sc.advance(sW, H, dt + 1, wq);
+            if ((warp & 3) == 0 && lane == 0)  // this warp's view (wq = 0) is the depth of the whole tile
+              s_nat[X][(v + 1) & 1] = (tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, dt + 1) + 7) / 8;
+            if (MODE == ATF_MODE_EXACT && H - sc.r_mid < zeroed_from) {
+              if (!wait_or_abort(bar(B_SFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 35; break; }
+              zero_q_down_to(H - sc.r_mid);
+            }
           }
         }
+        tc_wait_st();
+        tc_fence_before();
+        if (row == 0 && X == 1) ATF_STAMP(3 + 5 * X, 2 * v + h);
+#ifdef ATF_TRACE
+        if (X == 1 && lane == 0 && (warp & 3) > 0) ATF_STAMP((warp & 3), 2 * v + h);
+#endif
+        mbar_arrive(bar(B_PFULL + 2 * X + h));
       }
-      // zero the Q columns that stop being live in most cells at the next step
-      if (v + 1 < nX) {
-        sc.advance(sW, H, dt + 1, wq);
-        zero_q_down_to(H - sc.r_mid);
-      }
-      tc_wait_st();
-      tc_fence_before();
-      if (row == 0) ATF_STAMP(3 + 5 * X, v);
-      mbar_arrive(bar(B_PH1 + X));
     }
-
     if (ok && nX > 0) {
       if (!wait_or_abort(bar(B_OFULL + X), 0, abortp)) {
         ok = false;
