@@ -320,9 +320,9 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "achieved": executed / (pre_ms * 1e-3) / 1e12,
                      "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": executed / (pre_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
-                     # DRAM bytes of one launch: ncu capture at N = 32768 (511 MB) scaled by N (traffic is the
+                     # DRAM bytes of one launch: ncu capture at N = 32768 (513 MB) scaled by N (traffic is the
                      # repacked Q/K, V and O once each, linear in N); see profiles/
-                     "traffic": 511.2e6 * wl.N / 32768 if wl.name == "llama-3.2-3b" else None,
+                     "traffic": 513.4e6 * wl.N / 32768 if wl.name == "llama-3.2-3b" else None,
                      "kernel": "atf_prefill_kernel (+2 repack launches, <1% of the time)",
                      "peak_source": f"{pk['source']} sustained bf16 GEMM"},
         "roofline_decode": {"bound": "hbm", "achieved": dbytes / (dec_us * 1e-6) / 1e9, "peak": pk["hbm_gbs"],

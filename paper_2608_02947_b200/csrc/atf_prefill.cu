@@ -53,8 +53,11 @@ constexpr int PF_THREADS = 384;
 static_assert(128 * 72 + 256 * 216 <= PF_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag behind
 
-// Optional timeline tracing (compile with -DATF_TRACE): block (0,0,0) stamps %clock64 at a few
-// events per step into the first words of the repacked-K scratch tail.  Off in normal builds.
+// Optional timeline tracing (compile with -DATF_TRACE): one CTA stamps %clock64 at a few events
+// per half step into a caller-provided device buffer of 16 x 64 words: slots 6 / 7 = one softmax
+// warp of tile B before / after its wait for S, slots 10 / 13 = tile B's issuer when it sees P
+// and after it has committed the next S.  A stamp costs on the order of 100 clocks, so few are
+// kept.  Off in normal builds.
 #ifdef ATF_TRACE
 #define ATF_STAMP(slot, step) do { if (blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && (step) < 64) \
     P.trace[(slot) * 64 + (step)] = clock64(); } while (0)
@@ -411,9 +414,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (h == 0 && more) natoms = *reinterpret_cast<volatile int*>(&s_nat[X][(v + 1) & 1]);
           if (X == 1) ATF_STAMP(10, 2 * v + h);
           issue_pv(t, h, v == 0 && h == 0);
-          if (X == 1) ATF_STAMP(11, 2 * v + h);
           if (more) issue_qk(t + 1, h, natoms);
-          if (X == 1) ATF_STAMP(12, 2 * v + h);
           tc_commit(bar(B_SFULL + 2 * X + h));  // S(v + 1, h) is there, and every product before it is complete
           if (X == 1) ATF_STAMP(13, 2 * v + h);
         }
@@ -486,13 +487,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll 1
       for (int h = 0; h < 2; ++h) {
         const int c0 = h * HK;  // first key column of this half
+        if (X == 1 && lane == 0 && (warp & 3) == 2) ATF_STAMP(6, 2 * v + h);
         if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 32; break; }
         tc_fence_after();
-        if (row == 0) ATF_STAMP(0 + 5 * X, 2 * v + h);
-#ifdef ATF_TRACE
-        const bool tr1 = X == 1 && lane == 0 && (warp & 3) == 1;
-        if (tr1) ATF_STAMP(4, 2 * v + h);
-#endif
+        if (X == 1 && lane == 0 && (warp & 3) == 2) ATF_STAMP(7, 2 * v + h);
         float s[HK];
         if (natoms > 0) {
           tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
@@ -503,9 +501,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           for (int c = 0; c < HK; ++c) s[c] = 0.f;
         }
         
-#ifdef ATF_TRACE
-        if (tr1) ATF_STAMP(6, 2 * v + h);
-#endif
         // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
         //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
         //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
@@ -564,9 +559,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         if (h == 1) mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
 
-#ifdef ATF_TRACE
-        if (tr1) ATF_STAMP(14, 2 * v + h);
-#endif
         // ---- causal mask, dropped keys (exact mode: per cell) ----
         if (dt == 0 || zmax > zdrop) {
 #pragma unroll
@@ -614,9 +606,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           tc_wait_st();
         }
-#ifdef ATF_TRACE
-        if (tr1) ATF_STAMP(7, 2 * v + h);
-#endif
         const float neg_m = m_used == -INFINITY ? 0.f : -m_used * kScaleLog2;
         const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
         float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -637,9 +626,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           pk[c >> 1] = pack_bf16x2(x.x, x.y);
         }
         tc_st32(tS + c0, pk);
-#ifdef ATF_TRACE
-        if (tr1) ATF_STAMP(9, 2 * v + h);
-#endif
         {
           const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
           l_run = l_run * scale_o + ((a01.x + a01.y) + (a23.x + a23.y));
@@ -672,10 +658,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         tc_wait_st();
         tc_fence_before();
-        if (row == 0 && X == 1) ATF_STAMP(3 + 5 * X, 2 * v + h);
-#ifdef ATF_TRACE
-        if (X == 1 && lane == 0 && (warp & 3) > 0) ATF_STAMP((warp & 3), 2 * v + h);
-#endif
         mbar_arrive(bar(B_PFULL + 2 * X + h));
       }
     }
