@@ -166,6 +166,25 @@ def attention_rows(Q, K, V, W, rows):
     return O, LSE
 
 
+def attention_appended_rows(Qc, K, V, W, n0, rows=None):
+    """Appended rows (App. C, "The interval itself"; Sec. 7.3 runs prefill in such chunks): the
+    context already holds keys 0..n0-1; the Nq new rows sit at positions n0..n0+Nq-1 and see keys
+    0..n0+Nq-1.  Qc[Nq,d] rotated at those positions, K[Nk,d] rotated, V[Nk,d], Nk = n0 + Nq.
+    Each row is the row of the single-shot definition at its position.  `rows` indexes Qc.
+    Returns (O[len(rows), d], LSE[len(rows)]).
+    """
+    Nq, d = Qc.shape
+    assert K.shape[0] == n0 + Nq and V.shape[0] == n0 + Nq
+    rows = range(Nq) if rows is None else list(rows)
+    O = np.empty((len(rows), d), dtype=np.float64)
+    LSE = np.empty(len(rows), dtype=np.float64)
+    for j, i in enumerate(rows):
+        n = n0 + i
+        s = windowed_scores_row(Qc[i], K, W, n)
+        O[j], LSE[j] = _softmax_row(s, V[: n + 1])
+    return O, LSE
+
+
 def attention_gqa(Q, K, V, W, rows=None):
     """All heads: Q[B,Hq,N,d], K/V[B,Hkv,N,d]; query head hq reads KV head hq // (Hq/Hkv)."""
     B, Hq, N, d = Q.shape
@@ -236,6 +255,18 @@ def kept_terms_prefill(W: np.ndarray, N: int) -> int:
     """Terms kept over all rows 0..N-1 of one head."""
     n = np.arange(N, dtype=np.int64)[:, None]
     return int((np.minimum(np.asarray(W, dtype=np.int64)[None, :], n) + 1).sum(dtype=np.int64))
+
+
+def kept_terms_interval(W: np.ndarray, n0: int, n1: int) -> int:
+    """Terms kept over the rows n0..n1-1 (positions from 0) of one head: the appended-rows step
+    of App. C; [0, N) is the whole prefill, [L-1, L) the decode step."""
+    n = np.arange(n0, n1, dtype=np.int64)[:, None]
+    return int((np.minimum(np.asarray(W, dtype=np.int64)[None, :], n) + 1).sum(dtype=np.int64))
+
+
+def pruned_share_interval(W, d, n0, n1) -> float:
+    full = (d // 2) * (n1 * (n1 + 1) // 2 - n0 * (n0 + 1) // 2)
+    return 1.0 - kept_terms_interval(W, n0, n1) / full
 
 
 def kept_terms_decode(W: np.ndarray, L: int) -> int:
