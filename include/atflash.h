@@ -118,6 +118,24 @@ atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, 
                           int Hq, int Hkv, int64_t N, int d, const int64_t* table, int causal,
                           const atf_opts* opts, void* stream);
 
+/* Appended rows: the context already holds keys 0..N-Nq-1; the Nq new query rows sit at the
+ * positions N-Nq..N-1 and attend to all N keys (App. C, "The interval itself": the row interval
+ * [n0, n1] whose two endpoints are the whole prefill and the decode step; Sec. 7.3 runs the 1M
+ * prefill as such chunks).  Every row gets exactly what atf_prefill gives it at that position
+ * of a length-N prompt: a prefill cut into chunks is bit-identical to the single shot.
+ *   Q, O: dev bf16 [B, Hq, Nq, d];  LSE: dev fp32 [B, Hq, Nq] or NULL;
+ *   K, V: dev bf16 [B, Hkv, N, d], rotated at positions 0..N-1;  1 <= Nq <= N (else
+ *   ATF_ERR_INVALID_ARG).  table, causal, opts, workspace, errors: as atf_prefill; the table's
+ *   entries are clipped at N, the number of keys.  opts->kept_terms counts the Nq rows only.
+ *   Workspace: atf_workspace_bytes(ATF_OP_PREFILL, ..., N, d) is enough for any Nq <= N.       */
+atf_status atf_prefill_chunk(const void* Q, const void* K, const void* V, void* O, float* LSE,
+                             int B, int Hq, int Hkv, int64_t Nq, int64_t N, int d,
+                             const int64_t* table, int causal, void* stream);
+atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, void* O, float* LSE,
+                                int B, int Hq, int Hkv, int64_t Nq, int64_t N, int d,
+                                const int64_t* table, int causal, const atf_opts* opts,
+                                void* stream);
+
 /* Decode: one new query token per sequence against a contiguous KV cache (Sec. 5; the last
  * row of Fig. 3).  The cache already contains the new token; the query sits at position L-1,
  * so key m is at distance z = L-1-m.

@@ -52,6 +52,9 @@ def lib():
     L.atf_rope.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
     L.atf_prefill.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
+    L.atf_prefill_chunk.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i, vp]
+    L.atf_prefill_chunk_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i,
+                                       C.POINTER(_Opts), vp]
     L.atf_decode.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
     L.atf_decode_ex.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), C.POINTER(_Opts), vp]
     L.atf_kcache_pack.argtypes = [vp, vp, i, i, i64, i64, i64, i, vp]
@@ -65,7 +68,8 @@ def lib():
     L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
     L.atf_check_status.argtypes = [vp]
     L.atf_last_error.restype = C.c_char_p
-    for name in ("atf_window_table", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_decode", "atf_decode_ex",
+    for name in ("atf_window_table", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
+                 "atf_prefill_chunk_ex", "atf_decode", "atf_decode_ex",
                  "atf_kcache_pack",
                  "atf_bind_workspace", "atf_check_status"):
         getattr(L, name).restype = C.c_int
@@ -180,8 +184,10 @@ def _host_roundtrip(tensors):
 
 def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
                 O=None, LSE=None):
-    """Windowed causal attention.  Q [B,Hq,N,d], K/V [B,Hkv,N,d] bf16, already rotated.
+    """Windowed causal attention.  Q [B,Hq,Nq,d], K/V [B,Hkv,N,d] bf16, already rotated.
 
+    Nq == N is the whole prefill (atf_prefill_ex); Nq < N are appended rows: Q holds the last Nq
+    positions of the N-key context (atf_prefill_chunk_ex).
     Device tensors are used in place; host tensors are copied to the current CUDA device and
     the results copied back (host in -> host out).  Returns (O, LSE) (LSE None if not asked).
     """
@@ -190,21 +196,27 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
         Q, K, V = _host_roundtrip([Q, K, V])
     for t, nm in ((Q, "Q"), (K, "K"), (V, "V")):
         _dev_bf16(t, nm)
-    B, Hq, N, d = Q.shape
-    Hkv = K.shape[1]
+    B, Hq, Nq, d = Q.shape
+    Hkv, N = K.shape[1], K.shape[2]
     if K.shape != (B, Hkv, N, d) or V.shape != K.shape:
         raise AtfError(1, "K and V must be [B,Hkv,N,d] matching Q")
     if O is None:
         O = torch.empty_like(Q)
     if LSE is None and return_lse:
-        LSE = torch.empty((B, Hq, N), dtype=torch.float32, device=Q.device)
+        LSE = torch.empty((B, Hq, Nq), dtype=torch.float32, device=Q.device)
     ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL, B, Hq, Hkv, N, d), Q.device)
     tab, _keep = _table_ptr(table, d)
     o = _opts(mode, kept_terms, None)
     lse_ptr = C.c_void_p(LSE.data_ptr()) if LSE is not None else None
-    _check(lib().atf_prefill_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
-                                C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv, N, d, tab, 1 if causal else 0,
-                                C.byref(o) if o is not None else None, _stream(Q)))
+    if Nq == N:
+        _check(lib().atf_prefill_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                    C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+                                    C.byref(o) if o is not None else None, _stream(Q)))
+    else:
+        _check(lib().atf_prefill_chunk_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()),
+                                          C.c_void_p(V.data_ptr()), C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv,
+                                          Nq, N, d, tab, 1 if causal else 0,
+                                          C.byref(o) if o is not None else None, _stream(Q)))
     if on_host:
         return _to_pinned_host(O), (_to_pinned_host(LSE) if LSE is not None else None)
     return O, LSE

@@ -69,12 +69,14 @@ constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag 
 #endif
 struct PrefillParams {
   long long* trace;
-  const __nv_bfloat16* Qp;  // pair-interleaved copy of Q, [B*Hq, N, D]
+  const __nv_bfloat16* Qp;  // pair-interleaved copy of Q, [B*Hq, Nq, D]
   __nv_bfloat16* O;
   float* LSE;
   unsigned long long* kept;
   unsigned int* status;
-  int Hq, Hkv, N;
+  int Hq, Hkv;
+  int N;   // number of keys; positions 0..N-1
+  int Nq;  // number of query rows: the last Nq positions, n0 = N - Nq .. N-1 (Nq = N: whole prefill)
 };
 
 template <int D>
@@ -214,7 +216,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int npt = (P.N + 2 * T - 1) / (2 * T);
-  const int ip = npt - 1 - (int)blockIdx.x;  // longest rows first
+  const int ip = npt - 1 - (int)blockIdx.x;  // longest rows first; the grid stops at the pair holding row n0
+  const int n0 = P.N - P.Nq;
   const int hq = blockIdx.y, b = blockIdx.z;
   const int bhq = b * P.Hq + hq;
   const int bhk = b * P.Hkv + hq / (P.Hq / P.Hkv);
@@ -270,7 +273,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_expect_tx(bar(B_QFULL), 2 * SM::TILE);
       for (int x = 0; x < 2; ++x)
         for (int kb = 0; kb < NB; ++kb)
-          tma_load_3d(sQ + x * SM::TILE + kb * BLK_BYTES, &tmQ, bar(B_QFULL), kb * 64, (itA + x) * T, bhq);
+          // rows before n0 do not exist in Q: the (possibly negative) coordinate reads zero fill there
+          tma_load_3d(sQ + x * SM::TILE + kb * BLK_BYTES, &tmQ, bar(B_QFULL), kb * 64, (itA + x) * T - n0, bhq);
       TileSched sc;
       for (int t = 0; t < Tt; ++t) {
         const int j = itB - t;
@@ -433,7 +437,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int itX = X ? itB : itA;
     const int nX = X ? nB : nA;
     const int n = itX * T + row;
-    const bool row_ok = n < P.N;
+    const bool row_ok = n >= n0 && n < P.N;
+    const int64_t qrow = (int64_t)bhq * P.Nq + (row_ok ? n - n0 : 0);  // row of Q, O and LSE
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem_base + X * T + lane_off;
     const uint32_t tO = tmem_base + 2 * T + X * D + lane_off;
@@ -465,7 +470,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float m_used = -INFINITY, l_run = 0.f;  // m_used in raw score units; -inf until a live cell is seen
     unsigned long long cnt = 0;
     const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
-    const __nv_bfloat16* qsrc = P.Qp + ((int64_t)bhq * P.N + (row_ok ? n : 0)) * D;
+    const __nv_bfloat16* qsrc = P.Qp + qrow * D;
 
     for (int t = 0; t < Tt && ok; ++t) {
       const int v = X ? t : t - 1;  // step of this query tile = its tile distance to key tile t
@@ -670,7 +675,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     if (ok && nX > 0) {
       tc_fence_after();
       const float inv = 1.f / l_run;
-      __nv_bfloat16* orow = P.O + ((int64_t)bhq * P.N + n) * D;
+      __nv_bfloat16* orow = P.O + qrow * D;
 #pragma unroll
       for (int q4 = 0; q4 < D / 32; ++q4) {
         uint32_t o[32];
@@ -688,7 +693,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
         }
       }
-      if (P.LSE && row_ok) P.LSE[(int64_t)bhq * P.N + n] = (m_used * kScaleLog2 + log2f(l_run)) * 0.6931471805599453f;
+      if (P.LSE && row_ok) P.LSE[qrow] = (m_used * kScaleLog2 + log2f(l_run)) * 0.6931471805599453f;
       if (COUNT) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
@@ -743,7 +748,8 @@ template <int D>
 atf_status launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& P,
                           const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
   const int npt = (P.N + 2 * T - 1) / (2 * T);
-  dim3 grid(npt, P.Hq, B);
+  const int ip0 = (P.N - P.Nq) / (2 * T);  // first tile pair with a query row
+  dim3 grid(npt - ip0, P.Hq, B);
   const int smem = PrefillSmem<D>::DYN_BYTES;
 #define ATF_PF_LAUNCH(MODE_, COUNT_)                                                                        \
   do {                                                                                                      \
@@ -783,11 +789,15 @@ static void* getenv_trace_ptr() {
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d) {
   return ATF_WS_HEADER + repack_bytes(B, Hq, N, d) + repack_bytes(B, Hkv, N, d);
 }
+static size_t prefill_chunk_workspace_bytes(int B, int Hq, int Hkv, int64_t Nq, int64_t N, int d) {
+  return ATF_WS_HEADER + repack_bytes(B, Hq, Nq, d) + repack_bytes(B, Hkv, N, d);
+}
 
-extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq,
-                                     int Hkv, int64_t N, int d, const int64_t* table, int causal,
-                                     const atf_opts* opts, void* stream) {
+extern "C" atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B,
+                                           int Hq, int Hkv, int64_t Nq, int64_t N, int d, const int64_t* table,
+                                           int causal, const atf_opts* opts, void* stream) {
   if (!Q || !K || !V || !O) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: null pointer");
+  if (Nq < 1 || Nq > N) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: need 1 <= Nq <= N (got Nq = %lld, N = %lld)", (long long)Nq, (long long)N);
   if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: d must be 64 or 128 (got %d)", d);
   if (B < 1 || Hq < 1 || Hkv < 1 || N < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: bad shape");
   if (Hq % Hkv) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: Hq must be a multiple of Hkv");
@@ -804,18 +814,18 @@ extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V
 
   AtfWorkspace ws = atf_bound_workspace();
   if (opts && opts->workspace) ws = AtfWorkspace{opts->workspace, opts->workspace_bytes};
-  const size_t need = atf_prefill_workspace_bytes(B, Hq, Hkv, N, d);
+  const size_t need = prefill_chunk_workspace_bytes(B, Hq, Hkv, Nq, N, d);
   if (!ws.ptr) return atf_fail(ATF_ERR_WORKSPACE, "atf_prefill: no workspace bound");
   if (ws.bytes < need) return atf_fail(ATF_ERR_WORKSPACE, "atf_prefill: workspace has %zu bytes, needs %zu", ws.bytes, need);
   if ((uintptr_t)ws.ptr & 255) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: workspace must be 256-byte aligned");
 
   char* base = (char*)ws.ptr;
   __nv_bfloat16* Qp = (__nv_bfloat16*)(base + ATF_WS_HEADER);
-  __nv_bfloat16* Kp = (__nv_bfloat16*)(base + ATF_WS_HEADER + repack_bytes(B, Hq, N, d));
+  __nv_bfloat16* Kp = (__nv_bfloat16*)(base + ATF_WS_HEADER + repack_bytes(B, Hq, Nq, d));
   cudaStream_t s = (cudaStream_t)stream;
 
   {
-    const int64_t rows_q = (int64_t)B * Hq * N, rows_k = (int64_t)B * Hkv * N;
+    const int64_t rows_q = (int64_t)B * Hq * Nq, rows_k = (int64_t)B * Hkv * N;
     const int64_t bq = (rows_q * (d / 8) + 255) / 256, bk = (rows_k * (d / 8) + 255) / 256;
     if (bq > 0x7FFFFFFF) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: problem too large for the repack grid");
     atf_repack_kernel<<<(unsigned)bq, 256, 0, s>>>((const __nv_bfloat16*)Q, Qp, rows_q, d);
@@ -824,7 +834,7 @@ extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V
   }
 
   CUtensorMap tq, tk, tv;
-  if ((st = make_tile_map(&tq, Qp, (int64_t)B * Hq, N, d)) != ATF_OK) return st;
+  if ((st = make_tile_map(&tq, Qp, (int64_t)B * Hq, Nq, d)) != ATF_OK) return st;
   if ((st = make_tile_map(&tk, Kp, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
   if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
 
@@ -838,9 +848,22 @@ extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.N = (int)N;
+  P.Nq = (int)Nq;
   const bool count = P.kept != nullptr;
   return d == 64 ? launch_prefill<64>(tq, tk, tv, P, t, B, mode, count, s)
                  : launch_prefill<128>(tq, tk, tv, P, t, B, mode, count, s);
+}
+
+extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq,
+                                     int Hkv, int64_t N, int d, const int64_t* table, int causal,
+                                     const atf_opts* opts, void* stream) {
+  return atf_prefill_chunk_ex(Q, K, V, O, LSE, B, Hq, Hkv, N, N, d, table, causal, opts, stream);
+}
+
+extern "C" atf_status atf_prefill_chunk(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq,
+                                        int Hkv, int64_t Nq, int64_t N, int d, const int64_t* table, int causal,
+                                        void* stream) {
+  return atf_prefill_chunk_ex(Q, K, V, O, LSE, B, Hq, Hkv, Nq, N, d, table, causal, nullptr, stream);
 }
 
 extern "C" atf_status atf_prefill(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq,
