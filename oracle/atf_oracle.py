@@ -97,6 +97,49 @@ def window_table(base: float, d: int, k: float, N: int, scaling: dict | None = N
     return W, theta
 
 
+def window_table_family(base: float, d: int, N: int, scaling: dict | None = None, *, profile: str = "constant",
+                        k_hi: float = 2.0, k_lo: float | None = None, gamma: float = 1.0, beta: float = 0.0,
+                        cap: float | None = None, a: float = 0.0, nope_fraction: float = 0.0):
+    """The window family of App. A:  w_r = min(max(k_r * lambda'_r**gamma + a*(r+1)/(d/2), beta), cap),
+    then W_r = floor(min(w_r, N)) as in Eq. 3.
+
+    k_r is the retention profile over the pair index r = 0 (highest frequency) .. d/2-1:
+    "constant" k_hi; "arithmetic" falls from k_hi to k_lo by a constant amount per pair
+    (k_r = k_hi - (k_hi - k_lo)/(d/2 - 1) * r; 16 -> 2 is the paper's variable-k profile);
+    "geometric" falls by a constant ratio per pair (k_r = k_hi * (k_lo/k_hi)**(r/(d/2 - 1))).
+    cap = None means no ceiling other than N.  nope_fraction: that share of the pairs, taken
+    from the low-frequency end and rounded to the nearest whole pair, is position-free: its
+    rotation is removed (theta'_r = 0) and it is kept at every distance (W_r = N).
+    The default arguments are Eq. 3 with k = 2.  Returns (W int64[d/2], theta' float64[d/2]).
+    """
+    if profile not in ("constant", "arithmetic", "geometric"):
+        raise ValueError("unknown profile")
+    theta = effective_theta(base, d, scaling).copy()
+    h = d // 2
+    k_lo = k_hi if k_lo is None else k_lo
+    n_free = int(math.floor(nope_fraction * h + 0.5))
+    W = np.empty(h, dtype=np.int64)
+    for r in range(h):
+        if r >= h - n_free:
+            theta[r] = 0.0
+            W[r] = N
+            continue
+        lam = 2.0 * math.pi / theta[r]
+        if profile == "constant" or h == 1:
+            k_r = k_hi
+        elif profile == "arithmetic":
+            k_r = k_hi - (k_hi - k_lo) / (h - 1) * r
+        else:
+            k_r = k_hi * math.pow(k_lo / k_hi, r / (h - 1))
+        lam_g = lam if gamma == 1.0 else math.pow(lam, gamma)
+        w = k_r * lam_g + a * (r + 1) / h
+        w = max(w, beta)
+        if cap is not None:
+            w = min(w, cap)
+        W[r] = N if not (w < N) else int(math.floor(w))
+    return W, theta
+
+
 # ----------------------------------------------------------------------------------------
 # RoPE, half-split layout: pair r is dims (r, r + d/2)  (Sec. 3.1)
 # ----------------------------------------------------------------------------------------

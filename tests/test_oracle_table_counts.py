@@ -202,3 +202,62 @@ def test_coarse_counts_brute_force():
         assert orc.coarse_kept_terms_prefill(W, N, T, T, G) == total
         assert orc.coarse_kept_terms_decode(W, N, 4) == sum(
             h - min(h, (int((W < N - 1 - m).sum()) // 4) * 4) if (W >= N - 1 - m).any() else 0 for m in range(N))
+
+
+# ---- the window family of App. A ----
+
+def test_family_defaults_are_eq3():
+    for base, d, N, sc in ((1e6, 64, 8192, None), (5e5, 128, 131072, gen_llama3()), (1e7, 128, 1 << 20, None)):
+        for k in (2.0, 0.5, 64.0):
+            W, th = orc.window_table(base, d, k, N, sc)
+            Wf, thf = orc.window_table_family(base, d, N, sc, k_hi=k)
+            assert np.array_equal(W, Wf) and np.array_equal(th, thf)
+
+
+def gen_llama3():
+    return {"kind": "llama3", "factor": 32.0, "low_freq_factor": 1.0, "high_freq_factor": 4.0, "original_ctx": 8192}
+
+
+def test_family_reproduces_table2_pruned_shares():
+    g = GOLD["table2_qk_pruned_percent"]
+    cases = (("qwen2.5-0.5b_16384", 1e6, 64, 16384), ("qwen2.5-7b-1m_117000", 1e7, 128, 117000),
+             ("qwen2.5-7b-1m_169000", 1e7, 128, 169000))
+    for key, base, d, N in cases:
+        for name, want in g[key].items():
+            if name == "k2":
+                W, _ = orc.window_table_family(base, d, N, k_hi=2.0)
+            elif name == "variable_16_to_2":
+                W, _ = orc.window_table_family(base, d, N, profile="arithmetic", k_hi=16.0, k_lo=2.0)
+            else:
+                W, _ = orc.window_table_family(base, d, N, k_hi=64.0)
+            assert np.all(np.diff(W) >= 0)
+            assert round(100 * orc.pruned_share_prefill(W, d, N), 1) == want, (key, name)
+
+
+def test_family_special_cases():
+    base, d, N = 1e6, 64, 4096
+    h = d // 2
+    # sliding window: every pair the same width (k_r = 0, floor = W)
+    W, _ = orc.window_table_family(base, d, N, k_hi=0.0, beta=500.0)
+    assert np.array_equal(W, np.full(h, 500))
+    # linear window: k_r = 0 and the additive term a (r+1)/(d/2) alone
+    W, _ = orc.window_table_family(base, d, N, k_hi=0.0, a=1000.0)
+    assert np.array_equal(W, np.floor(1000.0 * (np.arange(h) + 1) / h).astype(np.int64))
+    # ceiling as a fraction of the sequence length, floor in tokens
+    W0, _ = orc.window_table(base, d, 2.0, N)
+    W, _ = orc.window_table_family(base, d, N, k_hi=2.0, beta=64.0, cap=0.25 * N)
+    assert np.array_equal(W, np.clip(W0, 64, N // 4))
+    # wavelength exponent
+    W, th = orc.window_table_family(base, d, N, k_hi=2.0, gamma=0.5)
+    assert np.array_equal(W, np.floor(np.minimum(2.0 * np.sqrt(2 * np.pi / th), N)).astype(np.int64))
+    # geometric profile: end points k_hi and k_lo, every ratio equal
+    Wg, th = orc.window_table_family(base, d, 1 << 40, profile="geometric", k_hi=16.0, k_lo=2.0)
+    kr = Wg / (2 * np.pi / th)
+    assert abs(kr[0] - 16.0) < 0.2 and abs(kr[-1] - 2.0) < 1e-6
+    assert np.allclose(kr[2:] / kr[1:-1], (2.0 / 16.0) ** (1.0 / (h - 1)), rtol=2e-2)
+    # position-free pairs: the lowest-frequency quarter keeps everything and is not rotated
+    W, th = orc.window_table_family(base, d, N, k_hi=2.0, nope_fraction=0.25)
+    assert np.all(W[-8:] == N) and np.all(th[-8:] == 0.0) and np.array_equal(W[:-8], W0[:-8])
+    x = np.random.default_rng(0).standard_normal((5, d))
+    y = orc.rope_half_split(x, th, pos0=1000, round_bf16=False)
+    assert np.array_equal(y[:, h - 8:h], x[:, h - 8:h]) and np.array_equal(y[:, d - 8:], x[:, d - 8:])
