@@ -94,6 +94,33 @@ typedef struct {
 atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_scaling* s,
                             int64_t* w_out, double* theta_out);
 
+/* The window family of App. A (its Eq. for w_r):
+ *   w_r = min(max(k_r * lambda'_r^gamma + a * (r+1)/(d/2), beta), cap),  W_r = floor(min(w_r, N)).
+ * k_r is the retention profile over the pair index r = 0 (highest frequency) .. d/2-1:
+ *   ATF_PROFILE_CONSTANT    k_r = k_hi;
+ *   ATF_PROFILE_ARITHMETIC  k_r = k_hi - (k_hi - k_lo)/(d/2-1) * r   (16 -> 2: the variable-k profile);
+ *   ATF_PROFILE_GEOMETRIC   k_r = k_hi * (k_lo/k_hi)^(r/(d/2-1)).
+ * cap <= 0 or INFINITY: no ceiling other than N.  nope_fraction: that share of the pairs, from the
+ * low-frequency end, rounded to the nearest whole pair, is position-free: theta_out[r] = 0 (atf_rope
+ * then leaves the pair unrotated) and w_out[r] = N.  {CONSTANT, k_hi = k, gamma = 1, beta = 0,
+ * cap = 0, a = 0, nope_fraction = 0} is atf_window_table, bit for bit.
+ * The table may come out non-monotone in r (e.g. a steep profile or a negative a); the attention
+ * entry points accept only non-decreasing tables and return ATF_ERR_UNSUPPORTED otherwise.
+ * Errors: as atf_window_table, plus ATF_ERR_INVALID_ARG for f NULL, an unknown profile, k_hi < 0,
+ * k_lo < 0 (k_lo <= 0 with the geometric profile), beta < 0, nope_fraction outside [0, 1], NaNs.  */
+enum { ATF_PROFILE_CONSTANT = 0, ATF_PROFILE_ARITHMETIC = 1, ATF_PROFILE_GEOMETRIC = 2 };
+typedef struct {
+  int profile;
+  double k_hi, k_lo;     /* k_lo is ignored by the constant profile */
+  double gamma;          /* wavelength exponent */
+  double beta;           /* floor, tokens */
+  double cap;            /* ceiling, tokens; <= 0 or INFINITY = none */
+  double a;              /* coefficient of the term linear in the pair index */
+  double nope_fraction;  /* share of position-free pairs at the low-frequency end */
+} atf_window_family;
+atf_status atf_window_table_family(double base, int d, int64_t N, const atf_scaling* s,
+                                   const atf_window_family* f, int64_t* w_out, double* theta_out);
+
 /* Half-split rotary embedding, in place (Sec. 3.1).
  *   X: dev bf16 [B, H, N, d]; row n is rotated by the angle (pos0 + n) * theta[r] in pair r:
  *   x'_r = x_r cos - x_{r+d/2} sin,  x'_{r+d/2} = x_{r+d/2} cos + x_r sin.

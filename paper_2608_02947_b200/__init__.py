@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     atf_prefill,
     atf_rope,
     atf_window_table,
+    atf_window_table_family,
     atf_workspace_bytes,
     ensure_workspace,
     lib,

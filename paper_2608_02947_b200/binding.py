@@ -49,6 +49,8 @@ def lib():
     L = C.CDLL(p)
     vp, i, i64, dbl = C.c_void_p, C.c_int, C.c_int64, C.c_double
     L.atf_window_table.argtypes = [dbl, i, dbl, i64, C.POINTER(_Scaling), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
+    L.atf_window_table_family.argtypes = [dbl, i, i64, C.POINTER(_Scaling), C.POINTER(_Family), C.POINTER(C.c_int64),
+                                          C.POINTER(C.c_double)]
     L.atf_rope.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
     L.atf_prefill.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
@@ -68,7 +70,7 @@ def lib():
     L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
     L.atf_check_status.argtypes = [vp]
     L.atf_last_error.restype = C.c_char_p
-    for name in ("atf_window_table", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
+    for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_decode", "atf_decode_ex",
                  "atf_kcache_pack",
                  "atf_bind_workspace", "atf_check_status"):
@@ -87,17 +89,40 @@ def llama3_scaling(factor=32.0, low_freq_factor=1.0, high_freq_factor=4.0, origi
             "high_freq_factor": high_freq_factor, "original_ctx": original_ctx}
 
 
+def _scaling_ref(scaling):
+    if scaling is None or scaling.get("kind", "none") == "none":
+        return None
+    kind = {"llama3": 1}.get(scaling["kind"], 99)
+    return C.byref(_Scaling(kind, float(scaling["factor"]), float(scaling["low_freq_factor"]),
+                            float(scaling["high_freq_factor"]), int(scaling["original_ctx"])))
+
+
 def atf_window_table(base, d, k, N, scaling=None):
     """Returns (W int64[d/2] tensor on the host, theta float64[d/2] tensor on the host)."""
     h = max(d // 2, 1)
     w = (C.c_int64 * h)()
     th = (C.c_double * h)()
-    sc = None
-    if scaling is not None and scaling.get("kind", "none") != "none":
-        kind = {"llama3": 1}.get(scaling["kind"], 99)
-        sc = C.byref(_Scaling(kind, float(scaling["factor"]), float(scaling["low_freq_factor"]),
-                              float(scaling["high_freq_factor"]), int(scaling["original_ctx"])))
-    _check(lib().atf_window_table(float(base), int(d), float(k), int(N), sc, w, th))
+    _check(lib().atf_window_table(float(base), int(d), float(k), int(N), _scaling_ref(scaling), w, th))
+    return torch.tensor(list(w), dtype=torch.int64), torch.tensor(list(th), dtype=torch.float64)
+
+
+class _Family(C.Structure):
+    _fields_ = [("profile", C.c_int), ("k_hi", C.c_double), ("k_lo", C.c_double), ("gamma", C.c_double),
+                ("beta", C.c_double), ("cap", C.c_double), ("a", C.c_double), ("nope_fraction", C.c_double)]
+
+
+_PROFILES = {"constant": 0, "arithmetic": 1, "geometric": 2}
+
+
+def atf_window_table_family(base, d, N, scaling=None, profile="constant", k_hi=2.0, k_lo=None, gamma=1.0, beta=0.0,
+                            cap=None, a=0.0, nope_fraction=0.0):
+    """The window family of App. A; same return as atf_window_table."""
+    h = max(d // 2, 1)
+    w = (C.c_int64 * h)()
+    th = (C.c_double * h)()
+    fam = _Family(_PROFILES.get(profile, 99), float(k_hi), float(k_hi if k_lo is None else k_lo), float(gamma),
+                  float(beta), 0.0 if cap is None else float(cap), float(a), float(nope_fraction))
+    _check(lib().atf_window_table_family(float(base), int(d), int(N), _scaling_ref(scaling), C.byref(fam), w, th))
     return torch.tensor(list(w), dtype=torch.int64), torch.tensor(list(th), dtype=torch.float64)
 
 

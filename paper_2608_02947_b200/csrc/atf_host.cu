@@ -104,6 +104,52 @@ atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_s
   return ATF_OK;
 }
 
+atf_status atf_window_table_family(double base, int d, int64_t N, const atf_scaling* s, const atf_window_family* f,
+                                   int64_t* w_out, double* theta_out) {
+  if (!f) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: f is NULL");
+  if (f->profile < ATF_PROFILE_CONSTANT || f->profile > ATF_PROFILE_GEOMETRIC)
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: unknown profile %d", f->profile);
+  if (!(f->k_hi >= 0.0)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: k_hi must be >= 0");
+  if (f->profile != ATF_PROFILE_CONSTANT && !(f->k_lo >= 0.0))
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: k_lo must be >= 0");
+  if (f->profile == ATF_PROFILE_GEOMETRIC && !(f->k_lo > 0.0 && f->k_hi > 0.0))
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: the geometric profile needs k_hi, k_lo > 0");
+  if (!(f->beta >= 0.0)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: beta must be >= 0");
+  if (!(f->nope_fraction >= 0.0 && f->nope_fraction <= 1.0))
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: nope_fraction must be in [0, 1]");
+  if (f->gamma != f->gamma || f->a != f->a || f->cap != f->cap)
+    return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table_family: NaN parameter");
+  // effective frequencies (and every argument check they share) from the Eq. 3 generator
+  double theta_local[ATF_MAX_PAIRS * 4];
+  if (d > 0 && d / 2 > ATF_MAX_PAIRS * 4)
+    return atf_fail(ATF_ERR_UNSUPPORTED, "atf_window_table_family: d/2 must be <= %d", ATF_MAX_PAIRS * 4);
+  atf_status st = atf_window_table(base, d, 1.0, N, s, w_out, theta_local);
+  if (st != ATF_OK) return st;
+  const double two_pi = 2.0 * M_PI;
+  const int h = d / 2;
+  const int n_free = (int)std::floor(f->nope_fraction * (double)h + 0.5);
+  const bool has_cap = f->cap > 0.0 && f->cap < INFINITY;
+  for (int r = 0; r < h; ++r) {
+    if (r >= h - n_free) {
+      if (theta_out) theta_out[r] = 0.0;
+      w_out[r] = N;
+      continue;
+    }
+    const double theta = theta_local[r];
+    if (theta_out) theta_out[r] = theta;
+    const double lam = two_pi / theta;
+    double k_r = f->k_hi;
+    if (h > 1 && f->profile == ATF_PROFILE_ARITHMETIC) k_r = f->k_hi - (f->k_hi - f->k_lo) / (double)(h - 1) * (double)r;
+    if (h > 1 && f->profile == ATF_PROFILE_GEOMETRIC) k_r = f->k_hi * std::pow(f->k_lo / f->k_hi, (double)r / (double)(h - 1));
+    const double lam_g = f->gamma == 1.0 ? lam : std::pow(lam, f->gamma);
+    double w = k_r * lam_g + f->a * (double)(r + 1) / (double)h;
+    w = w > f->beta ? w : f->beta;  // max(w, beta)
+    if (has_cap && f->cap < w) w = f->cap;
+    w_out[r] = (w < (double)N) ? (int64_t)std::floor(w) : N;
+  }
+  return ATF_OK;
+}
+
 atf_status atf_bind_workspace(void* dev_ptr, size_t bytes) {
   if (dev_ptr && ((uintptr_t)dev_ptr & 255)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_bind_workspace: pointer must be 256-byte aligned");
   if (dev_ptr && bytes < ATF_WS_HEADER) return atf_fail(ATF_ERR_WORKSPACE, "atf_bind_workspace: workspace smaller than its header");

@@ -70,3 +70,46 @@ def test_validation_returns_codes_without_a_device(atf):
     assert lib.atf_workspace_bytes(0, 1, 2, 1, 128, 96) == 0
     assert lib.atf_workspace_bytes(0, 1, 24, 8, 131072, 128) > 1 << 30
     assert lib.atf_kcache_tile_keys(128) == 64 and lib.atf_kcache_tile_keys(64) == 128
+
+
+FAMILY_CASES = [
+    dict(),  # Eq. 3 with k = 2
+    dict(k_hi=64.0),
+    dict(profile="arithmetic", k_hi=16.0, k_lo=2.0),
+    dict(profile="geometric", k_hi=16.0, k_lo=2.0),
+    dict(k_hi=2.0, gamma=0.5),
+    dict(k_hi=2.0, gamma=1.25, cap=3000.0),
+    dict(k_hi=2.0, beta=64.0, cap=0.25 * 8192),
+    dict(k_hi=0.0, beta=500.0),                # sliding window
+    dict(k_hi=0.0, a=1000.0),                  # linear window
+    dict(k_hi=1.0, a=300.0, nope_fraction=0.25),
+    dict(profile="arithmetic", k_hi=3.0, k_lo=8.0, a=-20.0, beta=5.0),
+]
+
+
+@pytest.mark.parametrize("base,d,N,sc", [(1e6, 64, 8192, None), (5e5, 128, 131072, LLAMA3_SCALING), (1e7, 128, 169000, None)])
+def test_host_family_table_equals_oracle(atf, base, d, N, sc):
+    for kw in FAMILY_CASES:
+        W, th = atf.atf_window_table_family(base, d, N, sc, **kw)
+        Wo, tho = orc.window_table_family(base, d, N, sc, **kw)
+        assert np.array_equal(W.numpy(), Wo), kw
+        assert np.array_equal(th.numpy(), tho), kw
+    W, th = atf.atf_window_table_family(base, d, N, sc, k_hi=2.0)
+    W2, th2 = atf.atf_window_table(base, d, 2.0, N, sc)
+    assert np.array_equal(W.numpy(), W2.numpy()) and np.array_equal(th.numpy(), th2.numpy())
+
+
+def test_family_validation_and_non_monotone_tables(atf):
+    lib = atf.lib()
+    for bad in (dict(profile="nope"), dict(k_hi=-1.0), dict(profile="geometric", k_hi=2.0, k_lo=0.0),
+                dict(beta=-1.0), dict(nope_fraction=1.5), dict(gamma=float("nan"))):
+        with pytest.raises(atf.AtfError):
+            atf.atf_window_table_family(1e6, 64, 4096, None, **bad)
+    assert lib.atf_window_table_family(1e6, 64, 4096, None, None, (C.c_int64 * 32)(), None) == 1
+    # a profile that rises faster than the wavelengths fall gives a table that is not monotone:
+    # the generator returns it, the attention entry points refuse it
+    W, _ = atf.atf_window_table_family(1e6, 64, 1 << 20, None, profile="geometric", k_hi=1e6, k_lo=1e-3)
+    assert np.any(np.diff(W.numpy()) < 0)
+    fake = C.c_void_p(4096)
+    tab = (C.c_int64 * 32)(*W.tolist())
+    assert lib.atf_prefill(fake, fake, fake, fake, None, 1, 2, 1, 1 << 20, 64, tab, 1, None) == 2
