@@ -194,12 +194,17 @@ def _opts(mode, kept_terms, lse, k_layout=ATF_KLAYOUT_ROWS):
     return o
 
 
-def _to_pinned_host(t):
-    """Device -> pinned host copy (a pageable destination would halve the PCIe rate)."""
-    h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
-    h.copy_(t, non_blocking=True)
+def _to_pinned_host(t, dst=None):
+    """Device -> host copy into `dst` (a host tensor of the same shape and dtype, ideally pinned and
+    reused by the caller: pinning a fresh buffer costs more than the copy) or into a new pinned
+    tensor (a pageable destination would halve the PCIe rate)."""
+    if dst is None:
+        dst = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+    elif dst.shape != t.shape or dst.dtype != t.dtype or dst.is_cuda:
+        raise AtfError(1, "host output tensor has the wrong shape, dtype or device")
+    dst.copy_(t, non_blocking=True)
     torch.cuda.current_stream(t.device).synchronize()
-    return h
+    return dst
 
 
 def _host_roundtrip(tensors):
@@ -214,11 +219,14 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
     Nq == N is the whole prefill (atf_prefill_ex); Nq < N are appended rows: Q holds the last Nq
     positions of the N-key context (atf_prefill_chunk_ex).
     Device tensors are used in place; host tensors are copied to the current CUDA device and
-    the results copied back (host in -> host out).  Returns (O, LSE) (LSE None if not asked).
+    the results copied back (host in -> host out; O / LSE, if given, are then host tensors that
+    receive the results).  Returns (O, LSE) (LSE None if not asked).
     """
     on_host = not Q.is_cuda
+    O_host = LSE_host = None
     if on_host:
         Q, K, V = _host_roundtrip([Q, K, V])
+        O_host, LSE_host, O, LSE = O, LSE, None, None
     for t, nm in ((Q, "Q"), (K, "K"), (V, "V")):
         _dev_bf16(t, nm)
     B, Hq, Nq, d = Q.shape
@@ -243,7 +251,7 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
                                           Nq, N, d, tab, 1 if causal else 0,
                                           C.byref(o) if o is not None else None, _stream(Q)))
     if on_host:
-        return _to_pinned_host(O), (_to_pinned_host(LSE) if LSE is not None else None)
+        return _to_pinned_host(O, O_host), (_to_pinned_host(LSE, LSE_host) if LSE is not None else None)
     return O, LSE
 
 
