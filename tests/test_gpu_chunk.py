@@ -127,3 +127,32 @@ def test_last_quarter_of_a_32k_prompt(atf):
         err = np.abs(gen.to_f64(O[0, hq, rows]) - O_ref)
         assert err.max() <= O_MAX and err.mean() <= O_MEAN, (hq, err.max(), err.mean())
         assert np.abs(L[0, hq, rows].double().cpu().numpy() - L_ref).max() <= LSE_TOL
+
+
+def test_128k_prompt_in_two_64k_chunks_is_the_single_shot(atf):
+    """The benchmark's shape run the way Sec. 7.3 runs long prompts: 64K chunks, each seeing the
+    keys that exist so far; bit-identical to the single-shot prefill, interval counts exact."""
+    w = gen.llama32_3b(131072, seed_off=6)
+    Q, K, V = gen.prefill_inputs(w, device="cuda")
+    Wt, theta = atf.atf_window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Wo, _ = orc.window_table(w.base, w.d, w.k, w.N, w.scaling)
+    atf.atf_rope(Q, theta)
+    atf.atf_rope(K, theta)
+    O_all, L_all = atf.atf_prefill(Q, K, V, table=Wt)
+    half = w.N // 2
+    # first chunk: 64K rows over 64K keys, its own table (clipped at 64K keys)
+    W1, _ = atf.atf_window_table(w.base, w.d, w.k, half, w.scaling)
+    kept1 = torch.zeros(w.Hq, dtype=torch.int64, device="cuda")
+    O1, L1 = atf.atf_prefill(Q[:, :, :half].contiguous(), K[:, :, :half].contiguous(), V[:, :, :half].contiguous(),
+                             table=W1, kept_terms=kept1)
+    # second chunk: the last 64K rows over all 128K keys
+    kept2 = torch.zeros(w.Hq, dtype=torch.int64, device="cuda")
+    O2, L2 = atf.atf_prefill(Q[:, :, half:].contiguous(), K, V, table=Wt, kept_terms=kept2)
+    torch.cuda.synchronize()
+    atf.binding.check_status()
+    assert torch.equal(O1.view(torch.int16), O_all[:, :, :half].contiguous().view(torch.int16))
+    assert torch.equal(O2.view(torch.int16), O_all[:, :, half:].contiguous().view(torch.int16))
+    assert torch.equal(L1, L_all[:, :, :half]) and torch.equal(L2, L_all[:, :, half:])
+    assert kept1.cpu().tolist() == [orc.kept_terms_interval(Wo, 0, half)] * w.Hq
+    assert kept2.cpu().tolist() == [orc.kept_terms_interval(Wo, half, w.N)] * w.Hq
+    assert kept1[0].item() + kept2[0].item() == orc.kept_terms_prefill(Wo, w.N)
