@@ -73,9 +73,11 @@ def kept_terms_decode(W, L):
     return sum(min(int(w), L - 1) + 1 for w in W)
 
 
-def prefill_flops(wl, W):
-    cells = wl.N * (wl.N + 1) // 2
-    executed = wl.B * wl.Hq * (4 * kept_terms_prefill(W, wl.N) + 2 * wl.d * cells)
+def prefill_flops(wl, W, n0=0):
+    """Executed and effective FLOPs of the query rows n0..N-1 (n0 = 0: the whole prefill)."""
+    cells = wl.N * (wl.N + 1) // 2 - n0 * (n0 + 1) // 2
+    kept = kept_terms_prefill(W, wl.N) - (kept_terms_prefill(W, n0) if n0 else 0)
+    executed = wl.B * wl.Hq * (4 * kept + 2 * wl.d * cells)
     effective = wl.B * wl.Hq * 4 * wl.d * cells
     return executed, effective
 
@@ -255,6 +257,25 @@ def run_ours(args):
         full_dec.append(b_.elapsed_time(c))
     full_pre_ms, full_dec_ms = statistics.median(full_pre), statistics.median(full_dec)  # same statistic as the windowed runs
 
+    # ---- the coarse mode (what the paper's ports time: tile-level live sets, no per-cell finish) and the
+    #      last half of the prompt as appended rows (App. C: the reduction is higher for late rows) ----
+    coarse_pre, half_pre = [], []
+    Qh = Qg[:, :, wl.N // 2:].contiguous()
+    Oh2 = torch.empty_like(Qh)
+    for _ in range(3):
+        a, b_, c = ev(), ev(), ev()
+        a.record()
+        atf.atf_prefill(Qg, Kg, V, table=W, mode=atf.ATF_MODE_COARSE, O=O, LSE=LSE)
+        b_.record()
+        atf.atf_prefill(Qh, Kg, V, table=W, O=Oh2, return_lse=False)
+        c.record()
+        torch.cuda.synchronize()
+        coarse_pre.append(a.elapsed_time(b_))
+        half_pre.append(b_.elapsed_time(c))
+    coarse_pre_ms, half_pre_ms = statistics.median(coarse_pre), statistics.median(half_pre)
+    del Qh, Oh2
+    half_exec, _ = prefill_flops(wl, Wl, n0=wl.N // 2)
+
     # ---- decode alone, cycling a KV pool of >= 512 MiB so that no read hits L2 from an earlier one ----
     kv_bytes = 2 * Kg.numel() * 2
     npool = max(2, math.ceil((512 << 20) / kv_bytes) + 1)
@@ -317,6 +338,8 @@ def run_ours(args):
         "prefill_effective_tflops": effective / (pre_ms * 1e-3) / 1e12,
         "prefill_full_ms": full_pre_ms, "prefill_speedup_vs_full": full_pre_ms / pre_ms,
         "prefill_full_tflops": effective / (full_pre_ms * 1e-3) / 1e12,
+        "prefill_coarse_ms": coarse_pre_ms, "prefill_coarse_speedup_vs_full": full_pre_ms / coarse_pre_ms,
+        "prefill_last_half_ms": half_pre_ms, "prefill_last_half_executed_tflops": half_exec / (half_pre_ms * 1e-3) / 1e12,
         "prefill_ceiling": effective / executed,
         "rope_ms": rope_ms, "work_ms": work_ms,
         "decode_us": dec_us, "decode_gbs": dbytes / (dec_us * 1e-6) / 1e9,
