@@ -364,7 +364,7 @@ def run_ours(args):
                             "kernel": "atf_decode_kernel", "peak_source": f"{pk['source']} copy bandwidth"},
         "e2e": {"value": executed / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "what": "atf_prefill on pinned host tensors: H2D of Q,K,V + kernels + D2H of O,LSE"},
+                "what": "atf_prefill on pinned host tensors = the C call atf_prefill_host: H2D of Q,K,V, kernels and D2H of O,LSE, overlapped chunk by chunk (16K rows) on three streams"},
         "gpu_launches": 6 * args.steps,
         "clocks": clocks,
         "cpu_baseline": cpu,

@@ -163,6 +163,27 @@ atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, voi
                                 const int64_t* table, int causal, const atf_opts* opts,
                                 void* stream);
 
+/* Prefill from and to HOST memory.  Same arguments and results as atf_prefill_ex, but Qh, Kh, Vh,
+ * Oh (bf16) and LSEh (fp32 or NULL) are HOST pointers, [B,H,N,d] / [B,Hq,N] dense.  The prompt is
+ * processed in chunks of chunk_rows query rows (0 = 16384) as successive appended-rows steps
+ * (see atf_prefill_chunk; bit-identical to the single shot for every chunk size), so that the
+ * host->device copy of the next chunk, the kernels of this one and the device->host copy of the
+ * previous one overlap on three streams.  Page-locked host buffers are needed for that overlap;
+ * pageable ones work but serialise.
+ *   dev_scratch: device memory, 256-byte aligned, at least atf_prefill_host_scratch_bytes(...)
+ *   bytes (the K/V caches, two Q / O / LSE chunk buffers and the prefill workspace; its first
+ *   bytes are a workspace header: binding it with atf_bind_workspace lets atf_check_status read
+ *   the kernels' status afterwards).  opts->workspace must be NULL.  The library allocates no
+ *   device memory; it creates two copy streams per device at the first call and keeps them.
+ *   The call returns once everything is queued; `stream` (and the host results) are complete when
+ *   the caller has synchronised `stream`.  Work already queued on `stream` is waited for.
+ * Errors: as atf_prefill_ex; ATF_ERR_WORKSPACE if the scratch is missing or too small.           */
+size_t atf_prefill_host_scratch_bytes(int B, int Hq, int Hkv, int64_t N, int d, int64_t chunk_rows);
+atf_status atf_prefill_host(const void* Qh, const void* Kh, const void* Vh, void* Oh, float* LSEh,
+                            int B, int Hq, int Hkv, int64_t N, int d, const int64_t* table,
+                            int causal, const atf_opts* opts, void* dev_scratch,
+                            size_t scratch_bytes, int64_t chunk_rows, void* stream);
+
 /* Decode: one new query token per sequence against a contiguous KV cache (Sec. 5; the last
  * row of Fig. 3).  The cache already contains the new token; the query sits at position L-1,
  * so key m is at distance z = L-1-m.

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     atf_decode_static,
     atf_kcache_pack,
     atf_prefill,
+    atf_prefill_host,
     atf_rope,
     atf_window_table,
     atf_window_table_family,

@@ -57,6 +57,10 @@ def lib():
     L.atf_prefill_chunk.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_chunk_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i,
                                        C.POINTER(_Opts), vp]
+    L.atf_prefill_host.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp,
+                                   C.c_size_t, i64, vp]
+    L.atf_prefill_host_scratch_bytes.argtypes = [i, i, i, i64, i, i64]
+    L.atf_prefill_host_scratch_bytes.restype = C.c_size_t
     L.atf_decode.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
     L.atf_decode_ex.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), C.POINTER(_Opts), vp]
     L.atf_kcache_pack.argtypes = [vp, vp, i, i, i64, i64, i64, i, vp]
@@ -71,7 +75,7 @@ def lib():
     L.atf_check_status.argtypes = [vp]
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
-                 "atf_prefill_chunk_ex", "atf_decode", "atf_decode_ex",
+                 "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
                  "atf_kcache_pack",
                  "atf_bind_workspace", "atf_check_status"):
         getattr(L, name).restype = C.c_int
@@ -224,6 +228,9 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
     """
     on_host = not Q.is_cuda
     O_host = LSE_host = None
+    if on_host and Q.shape[2] == K.shape[2]:
+        return atf_prefill_host(Q, K, V, table=table, causal=causal, mode=mode, kept_terms=kept_terms,
+                                return_lse=return_lse, O=O, LSE=LSE)
     if on_host:
         Q, K, V = _host_roundtrip([Q, K, V])
         O_host, LSE_host, O, LSE = O, LSE, None, None
@@ -252,6 +259,44 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
                                           C.byref(o) if o is not None else None, _stream(Q)))
     if on_host:
         return _to_pinned_host(O, O_host), (_to_pinned_host(LSE, LSE_host) if LSE is not None else None)
+    return O, LSE
+
+
+def atf_prefill_host(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
+                     O=None, LSE=None, chunk_rows=0, device=None):
+    """atf_prefill for HOST tensors (Q [B,Hq,N,d], K/V [B,Hkv,N,d] bf16, rotated): the C call copies,
+    computes and copies back chunk by chunk on three streams.  Pinned tensors overlap; O / LSE, if
+    given, are host tensors that receive the results (reuse pinned ones across calls).
+    Returns (O, LSE) on the host, complete."""
+    for t, nm in ((Q, "Q"), (K, "K"), (V, "V")):
+        if t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise AtfError(1, f"{nm} must be a contiguous host bf16 tensor")
+    B, Hq, N, d = Q.shape
+    Hkv = K.shape[1]
+    if K.shape != (B, Hkv, N, d) or V.shape != K.shape:
+        raise AtfError(1, "K and V must be [B,Hkv,N,d] matching Q")
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    if O is None:
+        O = torch.empty(Q.shape, dtype=torch.bfloat16, pin_memory=True)
+    if LSE is None and return_lse:
+        LSE = torch.empty((B, Hq, N), dtype=torch.float32, pin_memory=True)
+    for t, shp, dt in ((O, Q.shape, torch.bfloat16), (LSE, (B, Hq, N), torch.float32)):
+        if t is not None and (t.is_cuda or tuple(t.shape) != tuple(shp) or t.dtype != dt or not t.is_contiguous()):
+            raise AtfError(1, "host output tensor has the wrong shape, dtype or device")
+    need = int(lib().atf_prefill_host_scratch_bytes(B, Hq, Hkv, N, d, int(chunk_rows)))
+    if need == 0:
+        raise AtfError(1, "unsupported shape")
+    ws = ensure_workspace(need, device)  # the scratch starts with the workspace header the status check reads
+    tab, _keep = _table_ptr(table, d)
+    o = _opts(mode, kept_terms, None)
+    with torch.cuda.device(device):
+        stream = torch.cuda.current_stream(device)
+        _check(lib().atf_prefill_host(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                      C.c_void_p(O.data_ptr()), C.c_void_p(LSE.data_ptr()) if LSE is not None else None,
+                                      B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+                                      C.byref(o) if o is not None else None, C.c_void_p(ws.data_ptr()), ws.numel(),
+                                      int(chunk_rows), C.c_void_p(stream.cuda_stream)))
+        stream.synchronize()
     return O, LSE
 
 

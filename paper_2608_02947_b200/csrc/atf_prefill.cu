@@ -97,15 +97,18 @@ enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFUL
 constexpr int HK = T / 2;  // keys per half tile: S and P are produced and consumed in halves
 
 __global__ void __launch_bounds__(256)
-atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D) {
-  // one thread writes 8 consecutive output columns (4 pairs) of one row
+atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D,
+                  int64_t n_per_head, int64_t src_head_rows) {
+  // one thread writes 8 consecutive output columns (4 pairs) of one row; the source holds
+  // src_head_rows rows per head of which the first n_per_head are copied, the result is dense
   const int H = D / 2;
   const int per_row = D / 8;
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= rows * per_row) return;
   const int64_t row = gid / per_row;
   const int t = (int)(gid % per_row);
-  const __nv_bfloat16* src = X + row * D;
+  const int64_t head = row / n_per_head;
+  const __nv_bfloat16* src = X + (head * src_head_rows + (row - head * n_per_head)) * D;
   __align__(16) __nv_bfloat16 out[8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -730,11 +733,12 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // [BH, N, D] bf16 tensor, box = 64 columns x 128 rows x 1, 128-byte swizzle, zero fill outside.
-atf_status make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N, int D) {
+atf_status make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N, int D, int64_t head_rows = 0) {
+  if (head_rows == 0) head_rows = N;  // rows between two heads in memory (>= N)
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return atf_fail(ATF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)N * D * 2};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)head_rows * D * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)T, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -793,10 +797,13 @@ static size_t prefill_chunk_workspace_bytes(int B, int Hq, int Hkv, int64_t Nq, 
   return ATF_WS_HEADER + repack_bytes(B, Hq, Nq, d) + repack_bytes(B, Hkv, N, d);
 }
 
-extern "C" atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B,
-                                           int Hq, int Hkv, int64_t Nq, int64_t N, int d, const int64_t* table,
-                                           int causal, const atf_opts* opts, void* stream) {
+// kv_head_rows: rows between two heads of K and of V in memory (>= N; N for dense tensors).  A caller that
+// fills a full-length cache chunk by chunk passes the cache's length here and the rows present as N.
+atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq, int Hkv,
+                            int64_t Nq, int64_t N, int d, const int64_t* table, int causal, const atf_opts* opts,
+                            void* stream, int64_t kv_head_rows) {
   if (!Q || !K || !V || !O) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: null pointer");
+  if (kv_head_rows < N) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: K/V head stride smaller than N");
   if (Nq < 1 || Nq > N) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: need 1 <= Nq <= N (got Nq = %lld, N = %lld)", (long long)Nq, (long long)N);
   if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: d must be 64 or 128 (got %d)", d);
   if (B < 1 || Hq < 1 || Hkv < 1 || N < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: bad shape");
@@ -828,15 +835,15 @@ extern "C" atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const v
     const int64_t rows_q = (int64_t)B * Hq * Nq, rows_k = (int64_t)B * Hkv * N;
     const int64_t bq = (rows_q * (d / 8) + 255) / 256, bk = (rows_k * (d / 8) + 255) / 256;
     if (bq > 0x7FFFFFFF) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: problem too large for the repack grid");
-    atf_repack_kernel<<<(unsigned)bq, 256, 0, s>>>((const __nv_bfloat16*)Q, Qp, rows_q, d);
-    atf_repack_kernel<<<(unsigned)bk, 256, 0, s>>>((const __nv_bfloat16*)K, Kp, rows_k, d);
+    atf_repack_kernel<<<(unsigned)bq, 256, 0, s>>>((const __nv_bfloat16*)Q, Qp, rows_q, d, Nq, Nq);
+    atf_repack_kernel<<<(unsigned)bk, 256, 0, s>>>((const __nv_bfloat16*)K, Kp, rows_k, d, N, kv_head_rows);
     ATF_CUDA_CHECK(cudaGetLastError());
   }
 
   CUtensorMap tq, tk, tv;
   if ((st = make_tile_map(&tq, Qp, (int64_t)B * Hq, Nq, d)) != ATF_OK) return st;
   if ((st = make_tile_map(&tk, Kp, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
-  if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
+  if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, kv_head_rows)) != ATF_OK) return st;
 
   PrefillParams P;
   P.trace = (long long*)getenv_trace_ptr();
@@ -852,6 +859,12 @@ extern "C" atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const v
   const bool count = P.kept != nullptr;
   return d == 64 ? launch_prefill<64>(tq, tk, tv, P, t, B, mode, count, s)
                  : launch_prefill<128>(tq, tk, tv, P, t, B, mode, count, s);
+}
+
+extern "C" atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B,
+                                           int Hq, int Hkv, int64_t Nq, int64_t N, int d, const int64_t* table,
+                                           int causal, const atf_opts* opts, void* stream) {
+  return atf_prefill_impl(Q, K, V, O, LSE, B, Hq, Hkv, Nq, N, d, table, causal, opts, stream, N);
 }
 
 extern "C" atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int Hq,
