@@ -58,3 +58,24 @@ def test_host_path_rejects_device_tensors_and_small_scratch(atf):
     assert lib.atf_prefill_host_scratch_bytes(1, 2, 2, 1024, 128, 0) > 0
     assert lib.atf_prefill_host(fake, fake, fake, fake, None, 1, 2, 2, 1024, 128, None, 1, None, fake, 1024, 0, None) == 4
     assert lib.atf_prefill_host(fake, fake, fake, fake, None, 1, 2, 2, 1024, 128, None, 1, None, None, 0, 0, None) == 4
+
+
+def test_host_path_32k_llama_shape(atf):
+    """The benchmark's end-to-end route at a full-size shape: default chunking, pinned tensors."""
+    w = gen.llama32_3b(32768, seed_off=5)
+    Q, K, V = gen.prefill_inputs(w, device="cuda")
+    Wt, theta = atf.atf_window_table(w.base, w.d, w.k, w.N, w.scaling)
+    atf.atf_rope(Q, theta)
+    atf.atf_rope(K, theta)
+    O_dev, L_dev = atf.atf_prefill(Q, K, V, table=Wt)
+    torch.cuda.synchronize()
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    Oh = torch.empty(Q.shape, dtype=torch.bfloat16, pin_memory=True)
+    Lh = torch.empty(Q.shape[:3], dtype=torch.float32, pin_memory=True)
+    for _ in range(2):  # the second call reuses scratch, streams and result buffers
+        Oh.zero_()
+        O, L = atf.atf_prefill(Qh, Kh, Vh, table=Wt, O=Oh, LSE=Lh)
+        atf.binding.check_status()
+        assert O is Oh and L is Lh
+        assert torch.equal(O.view(torch.int16), O_dev.cpu().view(torch.int16))
+        assert torch.equal(L, L_dev.cpu())
