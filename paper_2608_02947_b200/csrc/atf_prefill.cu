@@ -584,9 +584,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
           }
           mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-#ifdef ATF_X_NOMAX
-          mx = s[0] + s[63];
-#endif
         }
         // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
         // (or when the row sees its first live cell)
@@ -625,10 +622,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (((c >> 1) & 3) < POLY_OF_4) {
             x = exp2_poly2(x);
           } else {
-#ifndef ATF_X_NOEXP
             x.x = ex2_approx(x.x);
             x.y = ex2_approx(x.y);
-#endif
           }
           acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
           pk[c >> 1] = pack_bf16x2(x.x, x.y);
