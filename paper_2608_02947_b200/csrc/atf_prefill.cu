@@ -47,10 +47,11 @@ constexpr int PF_THREADS = 384;
 #endif
 // Register budget.  The kernel is compiled for 168 registers per thread (65536 / 384, rounded
 // down to a multiple of 8), i.e. 64512 in use at launch.  The producer/MMA warpgroup then
-// shrinks to 72 and the two softmax warpgroups grow to 216: 128*72 + 256*216 = 64512.  The
+// shrinks to 56 and the two softmax warpgroups grow to 224: 128*56 + 256*224 = 64512 (measured: 72/216
+// is 0.5-2 % slower, 40/232 no better, 24/240 slower: the issuer thread starts to spill).  The
 // total after the change must not exceed the total at launch, or the growing warps wait for
 // registers that never come.
-static_assert(128 * 72 + 256 * 216 <= PF_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
+static_assert(128 * 56 + 256 * 224 <= PF_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag behind
 
 // Optional timeline tracing (compile with -DATF_TRACE): one CTA stamps %clock64 at a few events
@@ -271,7 +272,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   if (warp == ATF_PRODUCER_WARP) {
     // =============================== TMA producer ===============================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (lane == 0) {
       mbar_expect_tx(bar(B_QFULL), 2 * SM::TILE);
       for (int x = 0; x < 2; ++x)
@@ -302,7 +303,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     // warp 1 serves query tile B, warp 2 query tile A (one thread each).  A tcgen05.mma issue
     // blocks while the tensor pipe's queue is full and a lone thread runs its bookkeeping slowly,
     // so two issuers keep the pipe fed where one could not.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (lane == 0) {
       static_assert(KS == 2 && VS == 2, "stage selection below assumes two-stage rings");
       const int X = warp == 1 ? 1 : 0;
@@ -434,7 +435,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
   } else if (warp >= 4) {
     // =============================== softmax groups ===============================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     const int X = warp >= 8 ? 1 : 0;
     const int row = tid - (X ? 256 : 128);
     const int itX = X ? itB : itA;
@@ -699,7 +700,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
   } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   }
 
   if (fail_site) {
