@@ -361,6 +361,9 @@ def run_ours(args):
                             "unit": "GB/s", "frac": dbytes / (dec_us * 1e-6) / 1e9 / pk["hbm_gbs"],
                             # ncu: the row layout moves the whole K and V cache (128-byte DRAM lines)
                             "traffic": float(dbytes_full),
+                            # the same launch on the bytes it actually reads (= traffic)
+                            "achieved_bytes_read": dbytes_full / (dec_us * 1e-6) / 1e9,
+                            "frac_bytes_read": dbytes_full / (dec_us * 1e-6) / 1e9 / pk["hbm_gbs"],
                             "kernel": "atf_decode_kernel", "peak_source": f"{pk['source']} copy bandwidth"},
         "e2e": {"value": executed / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
