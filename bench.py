@@ -179,6 +179,27 @@ def run_ours(args):
                  atf.atf_workspace_bytes(1, wl.B, wl.Hq, wl.Hkv, wl.N, wl.d))
     atf.ensure_workspace(nbytes, dev)
 
+    if args.decode_group_major_only:
+        # for profiler captures of the decode kernel on the tiled group-major K cache: the cache is
+        # rotated and packed once, then `steps` decode launches; prints a short line
+        W, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+        W = atf.WindowTable(W)
+        atf.atf_rope(Qg, theta)
+        atf.atf_rope(Kg, theta)
+        qd.copy_(Qg[:, :, -1])
+        Kgm = atf.atf_kcache_pack(Kg)
+        a, b_ = ev(), ev()
+        for i in range(args.warmup + args.steps):
+            if i == args.warmup:
+                a.record()
+            atf.atf_decode(qd, Kgm, V, table=W, O=Od)
+        b_.record()
+        torch.cuda.synchronize()
+        atf.binding.check_status()
+        print(json.dumps({"decode_group_major_only": True, "workload": args.workload,
+                          "decode_us": a.elapsed_time(b_) * 1e3 / args.steps}))
+        return
+
     t_rope, t_pre, t_dec, t_step = [], [], [], []
 
     def step(timed):
@@ -430,6 +451,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--full-attention", action="store_true",
                     help="run the step with table = NULL (the library's own k = infinity mode)")
+    ap.add_argument("--decode-group-major-only", action="store_true",
+                    help="run only decode launches on the group-major K cache (for ncu captures)")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only the warm-up and timed steps (for ncu captures); prints a short line")
     args = ap.parse_args()
