@@ -30,9 +30,13 @@
 // pairs of the last step that are not live in every cell are zeroed in the CTA's own copy of
 // the Q tile; pairs only die as the distance grows, so the zeroing is monotone.
 // Coarse mode: depth = pairs live in any cell of the tile, rounded up to 8; diagonal tile full.
+//
+// Band schedule (Sec. 3.3: the active pairs of a tile are known statically; Sec. 5: distance
+// bands).  What a tile needs depends only on its tile distance and, in exact mode, on which
+// quarter of the query rows a warp owns, and it is the same for every CTA of a launch.  A small
+// pre-kernel therefore writes one 32-bit word per (tile distance, row quarter) once per launch;
+// every role of the main kernel reads its word one step ahead and does no schedule arithmetic.
 #include <cuda.h>
-
-#include <cstdlib>
 
 #include "atf_common.cuh"
 
@@ -54,22 +58,8 @@ constexpr int PF_THREADS = 384;
 static_assert(128 * 56 + 256 * 224 <= PF_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units the running max may lag behind
 
-// Optional timeline tracing (compile with -DATF_TRACE): one CTA stamps %clock64 at a few events
-// per half step into a caller-provided device buffer of 16 x 64 words: slots 6 / 7 = one softmax
-// warp of tile B before / after its wait for S, slots 10 / 13 = tile B's issuer when it sees P
-// and after it has committed the next S.  A stamp costs on the order of 100 clocks, so few are
-// kept.  Off in normal builds.
-#ifdef ATF_TRACE
-#define ATF_STAMP(slot, step) do { if (blockIdx.x == ATF_TRACE_BLOCK && blockIdx.y == 0 && blockIdx.z == 0 && (step) < 64) \
-    P.trace[(slot) * 64 + (step)] = clock64(); } while (0)
-#else
-#define ATF_STAMP(slot, step) do { } while (0)
-#endif
-#ifndef ATF_TRACE_BLOCK
-#define ATF_TRACE_BLOCK 0
-#endif
 struct PrefillParams {
-  long long* trace;
+  const uint32_t* sched;  // band schedule, [tile distance][row quarter], see SchedEntry
   const __nv_bfloat16* Qp;  // pair-interleaved copy of Q, [B*Hq, Nq, D]
   __nv_bfloat16* O;
   float* LSE;
@@ -120,34 +110,66 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
   *reinterpret_cast<uint4*>(Y + row * D + 8 * t) = *reinterpret_cast<const uint4*>(out);
 }
 
-// Live-pair bookkeeping for a tile at tile distance dt (tiles of 128, aligned at 0): cells
-// span distances [zmin, zmax].  w[] is non-decreasing, so the pairs reaching a distance z are
-// r >= r0(z), and r0 only grows with dt: the cursors are advanced, never rewound.
-struct TileSched {
-  // For the 32 query rows of softmax warp wq (0..3) of a tile at tile distance dt, the cells span
-  // distances [zlo, zhi].  r_any / r_all: first pair live in some / in every one of those cells.
-  // r_mid: first pair kept in the MMA for those rows, i.e. live at the distance from the warp's
-  // middle row to the tile's middle column (live in most of the warp's cells).  A pair kept by
-  // warp 0 (the rows nearest to the keys) is in the MMA depth of the whole tile; the rows of the
-  // other warps that do not keep it hold a zero in that column of Q.
-  int r_any = 0, r_mid = 0, r_all = 0;
-  __device__ __forceinline__ void advance(const int* w, int H, int dt, int wq) {
+// Band schedule word of (tile distance dt, row quarter wq), tiles of 128 aligned at 0.  The 32
+// query rows of quarter wq and the 128 keys of a tile at distance dt span the cell distances
+// [zlo, zhi].  w[] is non-decreasing, so the pairs reaching a distance z are r >= r0(z); counted
+// from the low-frequency end (p = h - r) the word holds
+//   p_all  pairs live in every one of those cells (w >= zhi),
+//   p_mid  pairs kept in the MMA for those rows: live at the distance from the quarter's middle
+//          row to the tile's middle column, i.e. in most cells (the few cells where such a pair
+//          is dead are taken back out; pairs live in only a minority of cells are left out and
+//          added where live),
+//   p_any  pairs live in some cell (w >= zlo),
+// and, the same in all four words of a tile distance (the view of quarter 0, whose rows are
+// nearest to the keys: a pair it keeps is in the MMA depth of the whole tile, the rows of the
+// other quarters that do not keep it hold a zero in that column of Q),
+//   natoms 16-column MMA steps of the S product, nkb 64-column K blocks to load,
+//   mask   the tile needs the per-cell causal / dropped-key test,
+//   plain  (per quarter) none of mask, per-cell finish, empty S or diagonal tile applies.
+// Coarse mode: every quarter gets quarter 0's word; depth = pairs live anywhere in the tile
+// rounded up to a group of 8, everything on the diagonal tile.
+struct SchedEntry {
+  int p_all, p_mid, p_any, natoms, nkb;
+  bool mask;
+  __device__ __forceinline__ explicit SchedEntry(uint32_t e)
+      : p_all(e & 127), p_mid((e >> 7) & 127), p_any((e >> 14) & 127), natoms((e >> 21) & 15), nkb((e >> 25) & 3),
+        mask((e >> 27) & 1) {}
+  // plain: the quarter's cells need neither the mask nor the per-cell finish, S is not empty and
+  // it is not the diagonal tile (so every row already has a reference maximum)
+  static __device__ __forceinline__ bool plain(uint32_t e) { return (e >> 28) & 1; }
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(128)
+atf_sched_kernel(const __grid_constant__ AtfTable table, int H, int ndt, uint32_t* __restrict__ out) {
+  const int dt = blockIdx.x * blockDim.x + threadIdx.x;
+  if (dt >= ndt) return;
+  const int Wmax = table.w[H - 1];
+  auto first_reaching = [&](int z) {  // first pair r with w[r] >= z
+    int r = 0;
+    while (r < H && table.w[r] < z) ++r;
+    return r;
+  };
+  uint32_t word[4];
+  int natoms = 0, nkb = 1;
+  for (int wq = 0; wq < 4; ++wq) {
     const int zlo = dt == 0 ? 0 : dt * T + 32 * wq - (T - 1);
     const int zhi = dt * T + 32 * wq + 31;
     const int zmid = dt == 0 ? 16 * wq + 15 : dt * T + 32 * wq - 48;
-    while (r_any < H && w[r_any] < zlo) ++r_any;
-    while (r_mid < H && w[r_mid] < zmid) ++r_mid;
-    while (r_all < H && w[r_all] < zhi) ++r_all;
+    const int p_any = H - first_reaching(zlo), p_mid = H - first_reaching(zmid), p_all = H - first_reaching(zhi);
+    if (wq == 0) {
+      const int depth = MODE == ATF_MODE_EXACT ? p_mid : (dt == 0 ? H : min(H, (p_any + 7) / 8 * 8));
+      natoms = (depth + 7) / 8;
+      const int ncols = MODE == ATF_MODE_EXACT ? 2 * p_any : 2 * depth;
+      nkb = max(1, (ncols + 63) / 64);
+    }
+    const bool mask = dt == 0 || (MODE == ATF_MODE_EXACT && (dt + 1) * T - 1 > Wmax);
+    const bool plain = !mask && natoms > 0 && dt > 0 && (MODE != ATF_MODE_EXACT || p_all == p_any);
+    word[wq] = (uint32_t)p_all | ((uint32_t)p_mid << 7) | ((uint32_t)p_any << 14) | ((uint32_t)natoms << 21) |
+               ((uint32_t)nkb << 25) | ((uint32_t)mask << 27) | ((uint32_t)plain << 28);
+    if (MODE != ATF_MODE_EXACT) word[wq] = word[0];
   }
-};
-// Pairs contracted by the MMA for a tile.  Exact mode: the pairs live in most cells (the few
-// cells where a pair of those is dead are subtracted afterwards; pairs live in only a minority
-// of the cells are left out and added where live).  Coarse mode: pairs live anywhere in the
-// tile, rounded up to a group of 8; everything on the diagonal tile.
-template <int MODE>
-__device__ __forceinline__ int tile_depth(int H, int p_any, int p_mid, int dt) {
-  if (MODE == ATF_MODE_EXACT) return p_mid;
-  return dt == 0 ? H : min(H, (p_any + 7) / 8 * 8);
+  *reinterpret_cast<uint4*>(out + 4 * dt) = make_uint4(word[0], word[1], word[2], word[3]);
 }
 // 2^x for a pair of values on the FMA pipe (x <= ~8; anything below -126, -inf included, gives
 // ~1e-38): round x to the nearest integer n with the 1.5*2^23 trick, evaluate a cubic minimax
@@ -177,6 +199,32 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+// P = 2^(s * scale + neg_m) for the 64 columns of one half of S, packed to bf16 pairs, and their
+// fp32 sum.  POLY of every 4 packed pairs take the polynomial (FMA pipe), the rest MUFU.
+template <int POLY>
+__device__ __forceinline__ float exp_half(float (&s)[64], float scale, float neg_m, uint32_t (&pk)[32]) {
+  const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(neg_m, neg_m);
+  float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+  for (int c = 0; c < 64; c += 2) {
+    float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
+    if (((c >> 1) & 3) < POLY) {
+      x = exp2_poly2(x);
+    } else {
+      x.x = ex2_approx(x.x);
+      x.y = ex2_approx(x.y);
+    }
+    acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
+    pk[c >> 1] = pack_bf16x2(x.x, x.y);
+  }
+  const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+  return (a01.x + a01.y) + (a23.x + a23.y);
+}
+// A half whose exponentials were taken against the row's existing reference maximum is redone
+// with its own maximum if their sum is not below this (it also catches infinities and NaNs).
+// Far below the fp32 range: O accumulates up to 2^20 such terms times |V|.
+constexpr float STALE_REF_GUARD = 1.8446744e19f;  // 2^64
 
 // Bounded wait that also gives up as soon as another role of the CTA has given up.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -216,7 +264,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + SM::BAR_OFF + 8 * B_COUNT);
   __shared__ int sW[ATF_MAX_PAIRS];
   __shared__ int s_abort;
-  __shared__ int s_nat[2][2];  // MMA depth of query tile X at its next step (by step parity), from its softmax group
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int npt = (P.N + 2 * T - 1) / (2 * T);
@@ -233,7 +280,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     mbar_init(bar(B_QFULL), 1);
     for (int i = 0; i < KS; ++i) {
       mbar_init(bar(B_KFULL + i), 1);
-      mbar_init(bar(B_KEMPTY + i), 256);  // every softmax thread, once it has seen both halves of S of its tile
+      mbar_init(bar(B_KEMPTY + i), 8);  // every softmax warp, once it has seen both halves of S of its tile
     }
     for (int i = 0; i < VS; ++i) {
       mbar_init(bar(B_VFULL + i), 1);
@@ -242,7 +289,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     for (int x = 0; x < 2; ++x) {
       for (int h = 0; h < 2; ++h) {
         mbar_init(bar(B_SFULL + 2 * x + h), 1);
-        mbar_init(bar(B_PFULL + 2 * x + h), 128);
+        mbar_init(bar(B_PFULL + 2 * x + h), 4);  // one arrival per softmax warp of the tile
       }
       mbar_init(bar(B_OFULL + x), 1);
       mbar_init(bar(B_QZ + x), 128);
@@ -279,14 +326,12 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int kb = 0; kb < NB; ++kb)
           // rows before n0 do not exist in Q: the (possibly negative) coordinate reads zero fill there
           tma_load_3d(sQ + x * SM::TILE + kb * BLK_BYTES, &tmQ, bar(B_QFULL), kb * 64, (itA + x) * T - n0, bhq);
-      TileSched sc;
+      uint32_t e_next = __ldg(P.sched);
       for (int t = 0; t < Tt; ++t) {
         const int j = itB - t;
-        const int dnear = max(t - 1, 0);  // the closer user of this key tile
-        sc.advance(sW, H, dnear, 0);
-        const int depth = tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, dnear);
-        const int ncols = MODE == ATF_MODE_EXACT ? 2 * (H - sc.r_any) : 2 * depth;
-        const int nkb = max(1, (ncols + 63) / 64);
+        // the K columns to load are those of the closer user of this key tile (distance max(t - 1, 0))
+        const int nkb = SchedEntry(e_next).nkb;
+        if (t >= 1 && t + 1 < Tt) e_next = __ldg(P.sched + 4 * t);
         const int ks = t % KS, vs = t % VS;
         if (!wait_or_abort(bar(B_KEMPTY + ks), ((t / KS) & 1) ^ 1, abortp)) { fail_site = 10; break; }
         mbar_expect_tx(bar(B_KFULL + ks), nkb * BLK_BYTES);
@@ -394,10 +439,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       if (!ok) fail_site = 20;
       for (int t = 0; t < toff && ok; ++t) ok = skip_v(t);
       int natoms = 0;
+      uint32_t e_next = 0;  // schedule word of the next step, fetched a step ahead
       if (ok && nX > 0) {
-        TileSched sc0;
-        sc0.advance(sW, H, 0, 0);
-        natoms = (tile_depth<MODE>(H, H - sc0.r_any, H - sc0.r_mid, 0) + 7) / 8;
+        natoms = SchedEntry(__ldg(P.sched)).natoms;
+        if (nX > 1) e_next = __ldg(P.sched + 4);
         ok = wait_or_abort(bar(B_KFULL + toff % KS), (toff / KS) & 1, abortp);
         if (ok) {
           tc_fence_after();
@@ -412,6 +457,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       for (int v = 0; v < nX && ok; ++v) {
         const int t = v + toff;
         const bool more = v + 1 < nX;
+        if (more) {
+          natoms = SchedEntry(e_next).natoms;
+          if (v + 2 < nX) e_next = __ldg(P.sched + 4 * (v + 2));
+        }
         ok = wait_or_abort(bar(B_VFULL + t % VS), (t / VS) & 1, abortp);
         if (more) ok = ok && wait_or_abort(bar(B_KFULL + (t + 1) % KS), ((t + 1) / KS) & 1, abortp);
         if (!ok) { fail_site = 22; break; }
@@ -419,12 +468,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int h = 0; h < 2; ++h) {
           if (!wait_or_abort(bar(B_PFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 23; break; }
           tc_fence_after();
-          if (h == 0 && more) natoms = *reinterpret_cast<volatile int*>(&s_nat[X][(v + 1) & 1]);
-          if (X == 1) ATF_STAMP(10, 2 * v + h);
           issue_pv(t, h, v == 0 && h == 0);
           if (more) issue_qk(t + 1, h, natoms);
           tc_commit(bar(B_SFULL + 2 * X + h));  // S(v + 1, h) is there, and every product before it is complete
-          if (X == 1) ATF_STAMP(13, 2 * v + h);
         }
         if (!ok) break;
         if (!more) tc_commit(bar(B_OFULL + X));
@@ -450,9 +496,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
     if (!ok) fail_site = 30;
-    // exact mode keeps/zeroes pairs per warp of rows; coarse mode decides per tile (warp 0's view)
-    const int wq = MODE == ATF_MODE_EXACT ? (warp & 3) : 0;
-    TileSched sc;
+    // exact mode keeps/zeroes pairs per quarter of the rows; coarse mode decides per tile (every
+    // quarter's schedule word is quarter 0's there)
+    const uint32_t* sched = P.sched + (warp & 3);
     int zeroed_from = H;  // pairs p >= zeroed_from are zero in the shared copy of Q_X
     auto zero_q_down_to = [&](int p_keep) {
       if (MODE == ATF_MODE_EXACT && p_keep < zeroed_from) {
@@ -465,9 +511,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         fence_proxy_async_smem();
       }
     };
+    uint32_t e_cur = 0;  // schedule word of the step at hand; the next one is fetched a step ahead
     if (ok) {
-      sc.advance(sW, H, 0, wq);
-      zero_q_down_to(H - sc.r_mid);
+      e_cur = __ldg(sched);
+      zero_q_down_to(SchedEntry(e_cur).p_mid);
       mbar_arrive(bar(B_QZ + X));
     }
 
@@ -476,30 +523,97 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int zdrop = MODE == ATF_MODE_EXACT ? Wmax : 0x7FFFFFFF;
     const __nv_bfloat16* qsrc = P.Qp + qrow * D;
 
-    for (int t = 0; t < Tt && ok; ++t) {
+    // The steps come in two kinds.  Far from the diagonal and from every window boundary a tile
+    // needs neither the mask nor the per-cell finish, and the row already has a reference maximum:
+    // the exponentials are taken against it directly (any reference gives the same softmax as
+    // long as nothing overflows), which saves the row maximum and its dependency in front of the
+    // exponentials.  Those "plain" steps are most of a long prompt and run in a loop of their own,
+    // kept small so that it stays in the instruction cache; everything else takes the general step
+    // below, one step at a time.
+    int t = 0;
+    int h_enter = 0;  // half at which the general step starts (1: the plain loop handed over its second half)
+    while (ok) {
+      // ---------------- plain steps ----------------
+      for (; t < Tt; ++t) {
+        const int v = X ? t : t - 1;
+        if (v < 1 || v >= nX || !SchedEntry::plain(e_cur)) break;
+        const uint32_t e_next = v + 1 < nX ? __ldg(sched + 4 * (v + 1)) : 0u;
+        const int ks = t % KS;
+        bool handed_over = false;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          const int c0 = h * HK;
+          if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 36; break; }
+          tc_fence_after();
+          float s[HK];
+          tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
+          tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
+          tc_wait_ld();
+          uint32_t pk[HK / 2];
+          const float lsum = exp_half<POLY_OF_4>(s, kScaleLog2, -m_used * kScaleLog2, pk);
+          if (__any_sync(0xffffffffu, !(lsum < STALE_REF_GUARD))) {
+            // S is still in tensor memory (P has not been stored): the general step redoes this half
+            h_enter = h;
+            handed_over = true;
+            break;
+          }
+          if (h == 1) {  // done with this K tile: both halves of S have been computed
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_KEMPTY + ks));
+          }
+          tc_st32(tS + c0, pk);
+          l_run += lsum;
+          if (h == 0) {
+            if (COUNT && row_ok) {  // every cell of the tile holds the same pairs (coarse: whole groups of 8, i.e. 8 per MMA step)
+              const SchedEntry E(e_cur);
+              cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? E.p_all : min(H, 8 * E.natoms)) * (unsigned long long)T;
+            }
+            if (MODE == ATF_MODE_EXACT && v + 1 < nX) {
+              const int p_keep = SchedEntry(e_next).p_mid;
+              if (p_keep < zeroed_from) {
+                if (!wait_or_abort(bar(B_SFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 37; break; }
+                zero_q_down_to(p_keep);
+              }
+            }
+          }
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(B_PFULL + 2 * X + h));
+        }
+        if (handed_over || !ok) break;
+        e_cur = e_next;
+      }
+      if (!ok) break;
+      // ---------------- one general step ----------------
+      if (t >= Tt) break;
+      do {
       const int v = X ? t : t - 1;  // step of this query tile = its tile distance to key tile t
       const bool active = v >= 0 && v < nX;
       const int ks = t % KS;
-      if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
       if (!active) {
-        mbar_arrive(bar(B_KEMPTY + ks));
-        continue;
+        // The arrival must fall into this use of the stage: the tile is loaded only after the
+        // previous use has been released by everyone.
+        if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
+        if (lane == 0) mbar_arrive(bar(B_KEMPTY + ks));
+        break;
       }
       const int dt = v;
-      const int zmax = (dt + 1) * T - 1;
-      const int p_any = H - sc.r_any, p_mid = H - sc.r_mid, p_all = H - sc.r_all;  // cursors already at dt
-      const int depth = tile_depth<MODE>(H, p_any, p_mid, dt);
-      const int natoms = (depth + 7) / 8;
+      const SchedEntry E(e_cur);
+      const uint32_t e_next = v + 1 < nX ? __ldg(sched + 4 * (v + 1)) : 0u;
+      const int p_any = E.p_any, p_mid = E.p_mid, p_all = E.p_all, natoms = E.natoms;
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
-      const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // the same over the warp's rows
+      const bool straddle = MODE == ATF_MODE_EXACT && p_all < p_any;
+      if (straddle) {
+        // the finish below reads K from shared memory
+        if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
+      }
 
 #pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
+      for (int h = h_enter; h < 2; ++h) {
         const int c0 = h * HK;  // first key column of this half
-        if (X == 1 && lane == 0 && (warp & 3) == 2) ATF_STAMP(6, 2 * v + h);
         if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 32; break; }
         tc_fence_after();
-        if (X == 1 && lane == 0 && (warp & 3) == 2) ATF_STAMP(7, 2 * v + h);
         float s[HK];
         if (natoms > 0) {
           tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
@@ -509,136 +623,125 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
           for (int c = 0; c < HK; ++c) s[c] = 0.f;
         }
-        
-        // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
-        //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
-        //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
-        //      no row of this warp has such a cell in it. ----
-        if (MODE == ATF_MODE_EXACT) {
-          for (int p = p_all; p < p_any; ++p) {
-            const int wp = sW[H - 1 - p];
-            const bool subtract = p < p_mid;
-            // distances of the warp's cells in chunk q (columns c0 + 32q ..) span
-            // [zw_lo - c0 - 32q - 31, zw_hi - c0 - 32q]
-            bool touched[2];
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const int hi = zw_hi - c0 - 32 * q, lo = zw_lo - c0 - 32 * q - 31;
-              touched[q] = subtract ? (hi > wp) : (lo <= wp && hi >= 0);
-            }
-            if (!touched[0] && !touched[1]) continue;
-            const uint32_t qq = *reinterpret_cast<const uint32_t*>(qsrc + 2 * p);
-            float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
-            if (subtract) {
-              q0 = -q0;
-              q1 = -q1;
-            }
-            const int col = 2 * p;
-            // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
-            const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
-            const int chunk = (col & 63) >> 3;
-            uint32_t base8[8];
-#pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
-            // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
-            // is formed on the FMA pipe as a saturated affine function of its column (the integer and
-            // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
-            const float jbf = (float)(zrow - wp - c0);
-            const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              if (touched[q]) {
-                // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
-                uint32_t kk[32];
-#pragma unroll
-                for (int cc = 0; cc < 32; ++cc) {
-                  const int c = q * 32 + cc;
-                  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + (c0 + c) * 128));
-                }
-#pragma unroll
-                for (int cc = 0; cc < 32; ++cc) {
-                  const int c = q * 32 + cc;
-                  const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
-                  const float coef = __saturatef(fmaf(ca, (float)c, cb));
-                  s[c] = fmaf(term, coef, s[c]);
+
+        uint32_t pk[HK / 2];  // P (bf16) goes over the first 32 columns of this half of S (column c holds keys 2c, 2c+1)
+        float lsum = 0.f, scale_o = 1.f;
+        {
+          // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their term back
+          //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not: add their
+          //      term in the cells inside the window.  Work in 32-column chunks and skip a chunk when
+          //      no row of this warp has such a cell in it. ----
+          if (straddle) {
+            const int zw_lo = dt * T + (warp & 3) * 32, zw_hi = zw_lo + 31;  // zrow over the warp's rows
+            for (int p = p_all; p < p_any; ++p) {
+              const int wp = sW[H - 1 - p];
+              const bool subtract = p < p_mid;
+              // distances of the warp's cells in chunk q (columns c0 + 32q ..) span
+              // [zw_lo - c0 - 32q - 31, zw_hi - c0 - 32q]
+              bool touched[2];
+  #pragma unroll
+              for (int q = 0; q < 2; ++q) {
+                const int hi = zw_hi - c0 - 32 * q, lo = zw_lo - c0 - 32 * q - 31;
+                touched[q] = subtract ? (hi > wp) : (lo <= wp && hi >= 0);
+              }
+              if (!touched[0] && !touched[1]) continue;
+              const uint32_t qq = *reinterpret_cast<const uint32_t*>(qsrc + 2 * p);
+              float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
+              if (subtract) {
+                q0 = -q0;
+                q1 = -q1;
+              }
+              const int col = 2 * p;
+              // shared-space address of this pair in key row 0 of the tile, one per swizzle phase of the row
+              const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+              const int chunk = (col & 63) >> 3;
+              uint32_t base8[8];
+  #pragma unroll
+              for (int k8 = 0; k8 < 8; ++k8) base8[k8] = kb32 + ((chunk ^ k8) << 4);
+              // Cells with column >= jb = zrow - wp are inside the pair's window.  The 0/1 factor of a cell
+              // is formed on the FMA pipe as a saturated affine function of its column (the integer and
+              // select pipes run at half rate): adding uses sat(c - jb + 1), taking back uses sat(jb - c).
+              const float jbf = (float)(zrow - wp - c0);
+              const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
+  #pragma unroll
+              for (int q = 0; q < 2; ++q) {
+                if (touched[q]) {
+                  // all 32 loads first (same address across the warp: a broadcast), then the arithmetic
+                  uint32_t kk[32];
+  #pragma unroll
+                  for (int cc = 0; cc < 32; ++cc) {
+                    const int c = q * 32 + cc;
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(base8[c & 7] + (c0 + c) * 128));
+                  }
+  #pragma unroll
+                  for (int cc = 0; cc < 32; ++cc) {
+                    const int c = q * 32 + cc;
+                    const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
+                    const float coef = __saturatef(fmaf(ca, (float)c, cb));
+                    s[c] = fmaf(term, coef, s[c]);
+                  }
                 }
               }
             }
           }
+          // ---- causal mask, dropped keys (exact mode: per cell) ----
+          if (E.mask) {
+  #pragma unroll
+            for (int c = 0; c < HK; ++c) {
+              const int z = zrow - c0 - c;
+              s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
+            }
+          }
+          float mx;
+          {
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+  #pragma unroll
+            for (int c = 0; c < HK; c += 8) {
+  #pragma unroll
+              for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
+            }
+            mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+          }
+          // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
+          // (or when the row sees its first live cell)
+          bool moved = false;
+          if (mx > m_used && (m_used == -INFINITY || (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD)) {
+            scale_o = m_used == -INFINITY ? 0.f : ex2_approx((m_used - mx) * kScaleLog2);
+            m_used = mx;
+            moved = !(v == 0 && h == 0);  // nothing has been accumulated before the first half
+          }
+          if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles
+            // every product issued so far must be complete: the issuer signals the other half's S
+            // barrier after each product (S(v, 1) follows P(v-1, 1) V; S(v+1, 0) follows P(v, 0) V)
+            const int vo = h == 0 ? v : v + 1;
+            if (!wait_or_abort(bar(B_SFULL + 2 * X + (h ^ 1)), vo & 1, abortp)) { ok = false; fail_site = 34; break; }
+            tc_fence_after();
+  #pragma unroll
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+              uint32_t o[32];
+              tc_ld32(tO + q4 * 32, o);
+              tc_wait_ld();
+  #pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
+              tc_st32(tO + q4 * 32, o);
+            }
+            tc_wait_st();
+          }
+          lsum = exp_half<POLY_OF_4>(s, kScaleLog2, m_used == -INFINITY ? 0.f : -m_used * kScaleLog2, pk);
         }
-        if (h == 1) mbar_arrive(bar(B_KEMPTY + ks));  // done with this K tile
+        if (h == 1) {  // done with this K tile: both halves of S have been computed
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(B_KEMPTY + ks));
+        }
 
-        // ---- causal mask, dropped keys (exact mode: per cell) ----
-        if (dt == 0 || zmax > zdrop) {
-#pragma unroll
-          for (int c = 0; c < HK; ++c) {
-            const int z = zrow - c0 - c;
-            s[c] = (z >= 0 && z <= zdrop) ? s[c] : -INFINITY;
-          }
-        }
-        float mx;
-        {
-          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-          for (int c = 0; c < HK; c += 8) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) m4[i] = fmaxf(m4[i], fmaxf(s[c + 2 * i], s[c + 2 * i + 1]));
-          }
-          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-        }
-        // lazy rescaling: the reference maximum only moves when it lags by more than the threshold
-        // (or when the row sees its first live cell)
-        float scale_o = 1.f;
-        bool moved = false;
-        if (mx > m_used && (m_used == -INFINITY || (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD)) {
-          scale_o = m_used == -INFINITY ? 0.f : ex2_approx((m_used - mx) * kScaleLog2);
-          m_used = mx;
-          moved = !(v == 0 && h == 0);  // nothing has been accumulated before the first half
-        }
-        if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles
-          // every product issued so far must be complete: the issuer signals the other half's S
-          // barrier after each product (S(v, 1) follows P(v-1, 1) V; S(v+1, 0) follows P(v, 0) V)
-          const int vo = h == 0 ? v : v + 1;
-          if (!wait_or_abort(bar(B_SFULL + 2 * X + (h ^ 1)), vo & 1, abortp)) { ok = false; fail_site = 34; break; }
-          tc_fence_after();
-#pragma unroll
-          for (int q4 = 0; q4 < D / 32; ++q4) {
-            uint32_t o[32];
-            tc_ld32(tO + q4 * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * scale_o);
-            tc_st32(tO + q4 * 32, o);
-          }
-          tc_wait_st();
-        }
-        const float neg_m = m_used == -INFINITY ? 0.f : -m_used * kScaleLog2;
-        const float2 sc2 = make_float2(kScaleLog2, kScaleLog2), nm2 = make_float2(neg_m, neg_m);
-        float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-        // ---- P (bf16) over the first 32 columns of this half of S (column c holds keys 2c and 2c+1) ----
-        uint32_t pk[HK / 2];
-#pragma unroll
-        for (int c = 0; c < HK; c += 2) {
-          float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
-          if (((c >> 1) & 3) < POLY_OF_4) {
-            x = exp2_poly2(x);
-          } else {
-            x.x = ex2_approx(x.x);
-            x.y = ex2_approx(x.y);
-          }
-          acc[(c >> 1) & 3] = __fadd2_rn(acc[(c >> 1) & 3], x);
-          pk[c >> 1] = pack_bf16x2(x.x, x.y);
-        }
         tc_st32(tS + c0, pk);
-        {
-          const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
-          l_run = l_run * scale_o + ((a01.x + a01.y) + (a23.x + a23.y));
-        }
-        
+        l_run = l_run * scale_o + lsum;
+
         if (h == 0) {
           if (COUNT && row_ok) {
             const int ncols = dt == 0 ? row + 1 : T;
-            cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : depth) * (unsigned long long)ncols;
+            // coarse mode: the tile's depth is whole groups of 8 pairs, i.e. 8 per MMA step
+            cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : min(H, 8 * natoms)) * (unsigned long long)ncols;
             if (MODE == ATF_MODE_EXACT) {
               for (int p = p_all; p < p_any; ++p) {
                 const int wp = sW[H - 1 - p];
@@ -650,20 +753,23 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           // Zero the Q columns that stop being live in most cells at the next step.  S(v + 1, 0) is
           // issued once this half of P is signalled, so the zeroing has to happen here; S(v, 1) still
           // needs the columns, so wait until it has been computed (it was issued long ago).
-          if (v + 1 < nX) {
-            sc.advance(sW, H, dt + 1, wq);
-            if ((warp & 3) == 0 && lane == 0)  // this warp's view (wq = 0) is the depth of the whole tile
-              s_nat[X][(v + 1) & 1] = (tile_depth<MODE>(H, H - sc.r_any, H - sc.r_mid, dt + 1) + 7) / 8;
-            if (MODE == ATF_MODE_EXACT && H - sc.r_mid < zeroed_from) {
+          if (MODE == ATF_MODE_EXACT && v + 1 < nX) {
+            const int p_keep = SchedEntry(e_next).p_mid;
+            if (p_keep < zeroed_from) {
               if (!wait_or_abort(bar(B_SFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 35; break; }
-              zero_q_down_to(H - sc.r_mid);
+              zero_q_down_to(p_keep);
             }
           }
         }
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar(B_PFULL + 2 * X + h));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_PFULL + 2 * X + h));
       }
+      e_cur = e_next;
+      } while (false);
+      ++t;
+      h_enter = 0;
     }
     if (ok && nX > 0) {
       if (!wait_or_abort(bar(B_OFULL + X), 0, abortp)) {
@@ -776,21 +882,15 @@ size_t repack_bytes(int B, int H, int64_t N, int d) {
 
 atf_status atf_validate_table(const char* who, const int64_t* table, int d, int64_t N, AtfTable* out);
 
-// With -DATF_TRACE the caller passes a device buffer address for the timeline in ATF_TRACE_PTR.
-static void* getenv_trace_ptr() {
-#ifdef ATF_TRACE
-  const char* e = getenv("ATF_TRACE_PTR");
-  return e ? (void*)strtoull(e, nullptr, 0) : nullptr;
-#else
-  return nullptr;
-#endif
-}
+// band schedule: one 16-byte record per tile distance a launch over N keys can meet
+static int sched_entries(int64_t N) { return 2 * (int)((N + 2 * T - 1) / (2 * T)) + 1; }
+static size_t sched_bytes(int64_t N) { return ((size_t)sched_entries(N) * 16 + 255) & ~(size_t)255; }
 
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d) {
-  return ATF_WS_HEADER + repack_bytes(B, Hq, N, d) + repack_bytes(B, Hkv, N, d);
+  return ATF_WS_HEADER + sched_bytes(N) + repack_bytes(B, Hq, N, d) + repack_bytes(B, Hkv, N, d);
 }
 static size_t prefill_chunk_workspace_bytes(int B, int Hq, int Hkv, int64_t Nq, int64_t N, int d) {
-  return ATF_WS_HEADER + repack_bytes(B, Hq, Nq, d) + repack_bytes(B, Hkv, N, d);
+  return ATF_WS_HEADER + sched_bytes(N) + repack_bytes(B, Hq, Nq, d) + repack_bytes(B, Hkv, N, d);
 }
 
 // kv_head_rows: rows between two heads of K and of V in memory (>= N; N for dense tensors).  A caller that
@@ -823,9 +923,18 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
   if ((uintptr_t)ws.ptr & 255) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: workspace must be 256-byte aligned");
 
   char* base = (char*)ws.ptr;
-  __nv_bfloat16* Qp = (__nv_bfloat16*)(base + ATF_WS_HEADER);
-  __nv_bfloat16* Kp = (__nv_bfloat16*)(base + ATF_WS_HEADER + repack_bytes(B, Hq, Nq, d));
+  uint32_t* sched = (uint32_t*)(base + ATF_WS_HEADER);
+  __nv_bfloat16* Qp = (__nv_bfloat16*)(base + ATF_WS_HEADER + sched_bytes(N));
+  __nv_bfloat16* Kp = (__nv_bfloat16*)(base + ATF_WS_HEADER + sched_bytes(N) + repack_bytes(B, Hq, Nq, d));
   cudaStream_t s = (cudaStream_t)stream;
+
+  {
+    const int ndt = sched_entries(N);
+    if (mode == ATF_MODE_EXACT)
+      atf_sched_kernel<ATF_MODE_EXACT><<<(ndt + 127) / 128, 128, 0, s>>>(t, d / 2, ndt, sched);
+    else
+      atf_sched_kernel<ATF_MODE_COARSE><<<(ndt + 127) / 128, 128, 0, s>>>(t, d / 2, ndt, sched);
+  }
 
   {
     const int64_t rows_q = (int64_t)B * Hq * Nq, rows_k = (int64_t)B * Hkv * N;
@@ -842,7 +951,7 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
   if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, kv_head_rows)) != ATF_OK) return st;
 
   PrefillParams P;
-  P.trace = (long long*)getenv_trace_ptr();
+  P.sched = sched;
   P.Qp = Qp;
   P.O = (__nv_bfloat16*)O;
   P.LSE = LSE;
