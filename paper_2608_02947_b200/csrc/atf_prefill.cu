@@ -17,11 +17,14 @@
 //   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one query row per thread:
 //               read S, finish the window rule, mask, online softmax with lazy rescaling of
 //               O, write P (bf16) over S in tensor memory.
-// A key tile is processed as two halves of 64 keys.  Each half of a query tile's 128 S columns
-// is a buffer of its own: when the softmax group has turned S(v, h) into P(v, h) the issuer
-// runs O += P(v, h) V(half h) and then S(v + 1, h) into the same columns, while the group is
-// already working on the other half.  The softmax groups, which are the busiest unit of the
-// kernel (one MUFU exponential per cell), so never wait for a product that is not yet issued.
+// S_X of a (query tile, key tile) pair is one 128 x 128 x depth product (a 64-key product costs the
+// tensor pipe as much as a 128-key one).  The softmax group turns it into P in two halves of 64
+// keys and signals each half, so O_X += P(half 0) V runs while the group works on half 1; after
+// O_X += P(half 1) V the issuer writes the next S_X over the same columns.  While a query tile
+// waits for that, the warps of the other query tile have the schedulers and the MUFU unit to
+// themselves; the two issuers hand each other a token so that their closing batches (the second
+// O product and the next S) reach the tensor pipe one after the other, which keeps the two
+// query tiles in alternation instead of working and waiting at the same time.
 //
 // Exact mode (the per-term definition).  For a tile at tile distance D the cells span
 // distances [z_min, z_max].  Pairs with w >= z_max are live in every cell: they are the MMA
@@ -48,6 +51,9 @@ constexpr int KS = 2, VS = 2;       // ring depths
 constexpr int PF_THREADS = 384;
 #ifndef ATF_PRODUCER_WARP
 #define ATF_PRODUCER_WARP 0
+#endif
+#ifndef ATF_ORDER_BATCHES
+#define ATF_ORDER_BATCHES 1
 #endif
 // Register budget.  The kernel is compiled for 168 registers per thread (65536 / 384, rounded
 // down to a multiple of 8), i.e. 64512 in use at launch.  The producer/MMA warpgroup then
@@ -82,9 +88,11 @@ struct PrefillSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for 1024-byte alignment
 };
 // barrier slots (8 bytes each) inside the BAR area
-// B_SFULL / B_PFULL: slot + 2 * X + h for query tile X (0 = A, 1 = B) and key half h of the tile
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 13, B_OFULL = 17,
-       B_QZ = 19, B_COUNT = 21 };
+// B_SFULL / B_PV0 / B_OFULL / B_QZ: slot + X for query tile X (0 = A, 1 = B); B_PFULL: slot + 2 * X + h
+// for key half h of the tile.  B_PV0: the product O_X += P(half 0) V of the step is complete.
+// B_ORDER + X: issuer X has issued the closing batch of its step on the current key tile.
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PV0 = 11, B_PFULL = 13,
+       B_OFULL = 17, B_QZ = 19, B_ORDER = 21, B_COUNT = 23 };
 constexpr int HK = T / 2;  // keys per half tile: S and P are produced and consumed in halves
 
 __global__ void __launch_bounds__(256)
@@ -251,7 +259,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   constexpr int H = D / 2;
   constexpr int NB = D / 64;
   constexpr uint32_t TMEM_COLS = 512;
-  constexpr uint32_t IDESC_QK = make_idesc_bf16(128, HK, 0, 0);
+  constexpr uint32_t IDESC_QK = make_idesc_bf16(128, T, 0, 0);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(128, D, 0, 1);
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
 
@@ -287,10 +295,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_init(bar(B_VEMPTY + i), 2);  // one arrival per MMA issuer
     }
     for (int x = 0; x < 2; ++x) {
-      for (int h = 0; h < 2; ++h) {
-        mbar_init(bar(B_SFULL + 2 * x + h), 1);
-        mbar_init(bar(B_PFULL + 2 * x + h), 4);  // one arrival per softmax warp of the tile
-      }
+      mbar_init(bar(B_SFULL + x), 1);
+      mbar_init(bar(B_PV0 + x), 1);
+      mbar_init(bar(B_ORDER + x), 1);
+      for (int h = 0; h < 2; ++h) mbar_init(bar(B_PFULL + 2 * x + h), 4);  // one arrival per softmax warp of the tile
       mbar_init(bar(B_OFULL + x), 1);
       mbar_init(bar(B_QZ + x), 128);
     }
@@ -361,11 +369,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const uint64_t dK0 = make_smem_desc_sw128(sK, 16, 1024), dK1 = make_smem_desc_sw128(sK + SM::TILE, 16, 1024);
       const uint64_t dV0 = make_smem_desc_sw128(sV, BLK_BYTES, 1024),
                      dV1 = make_smem_desc_sw128(sV + SM::TILE, BLK_BYTES, 1024);
-      // S_X(half h) = Q_X K(tile, keys 64h..64h+63)^T over natoms 16-column steps, into columns
-      // [64h, 64h+64) of the tile's S region; then signal the softmax group.
-      auto issue_qk = [&](int tile, int h, int natoms) {
-        const uint64_t k0 = ((tile & 1) ? dK1 : dK0) + (uint64_t)(h * 512);
-        const uint32_t tSx = tmem_base + X * T + h * HK;
+      // S_X = Q_X K(tile)^T over natoms 16-column steps, into the tile's 128 S columns.
+      auto issue_qk = [&](int tile, int natoms) {
+        const uint64_t k0 = (tile & 1) ? dK1 : dK0;
+        const uint32_t tSx = tmem_base + X * T;
         asm volatile(
             "{\n\t"
             ".reg .pred pf, p0, p1, p2, p3, p4, p5, p6, p7;\n\t"
@@ -422,11 +429,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             ::"r"(tOx), "r"(tPx), "l"(v0), "r"(IDESC_PV), "r"((uint32_t)(first ? 1 : 0))
             : "memory");
       };
-      // Each half of a query tile's S region is its own buffer: as soon as the softmax group has
-      // turned S(v, h) into P(v, h), the issuer runs O += P(v, h) V and then S(v + 1, h) into the
-      // same columns (the tensor pipe executes one thread's products in issue order), while the
-      // group is already working on the other half.  The softmax groups therefore never wait
-      // for the tensor pipe as long as it keeps up.
+      // Per step: O += P(half 0) V as soon as the softmax group has signalled that half (it is then
+      // working on half 1), O += P(half 1) V, and the next S over the same columns (the tensor pipe
+      // executes one thread's products in issue order).
       // A V stage is released by one arrival per issuer; an issuer that has no use for a key
       // tile still accounts for it, once the tile has been loaded (so that the arrival falls
       // into the right phase of the barrier).
@@ -446,10 +451,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ok = wait_or_abort(bar(B_KFULL + toff % KS), (toff / KS) & 1, abortp);
         if (ok) {
           tc_fence_after();
-          issue_qk(toff, 0, natoms);
-          tc_commit(bar(B_SFULL + 2 * X));
-          issue_qk(toff, 1, natoms);
-          tc_commit(bar(B_SFULL + 2 * X + 1));
+          issue_qk(toff, natoms);
+          tc_commit(bar(B_SFULL + X));
         } else {
           fail_site = 21;
         }
@@ -464,16 +467,33 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ok = wait_or_abort(bar(B_VFULL + t % VS), (t / VS) & 1, abortp);
         if (more) ok = ok && wait_or_abort(bar(B_KFULL + (t + 1) % KS), ((t + 1) / KS) & 1, abortp);
         if (!ok) { fail_site = 22; break; }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (!wait_or_abort(bar(B_PFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 23; break; }
-          tc_fence_after();
-          issue_pv(t, h, v == 0 && h == 0);
-          if (more) issue_qk(t + 1, h, natoms);
-          tc_commit(bar(B_SFULL + 2 * X + h));  // S(v + 1, h) is there, and every product before it is complete
+        if (!wait_or_abort(bar(B_PFULL + 2 * X), v & 1, abortp)) { ok = false; fail_site = 23; break; }
+        tc_fence_after();
+        issue_pv(t, 0, v == 0);
+        tc_commit(bar(B_PV0 + X));
+        if (!wait_or_abort(bar(B_PFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 23; break; }
+        // The closing batches of the two query tiles go to the tensor pipe in a fixed order, tile B's
+        // for key tile t, tile A's for key tile t, tile B's for t + 1, ...  Issued at the same time
+        // they would interleave and both finish late, and the two softmax groups would then work and
+        // wait in step with each other; one after the other, each group works while the other waits.
+        // A batch is announced only where the other issuer waits for it.
+        if (ATF_ORDER_BATCHES) {
+          const bool other_before = X == 0 ? t < nB : (t >= 2 && t - 1 <= nA);  // tile B's batch of t / tile A's of t - 1
+          const int tp = X == 0 ? t : t - 1;                                  // its key tile: announcements start at 1
+          if (other_before && !wait_or_abort(bar(B_ORDER + (X ^ 1)), (tp - 1) & 1, abortp)) { ok = false; fail_site = 26; break; }
         }
-        if (!ok) break;
-        if (!more) tc_commit(bar(B_OFULL + X));
+        tc_fence_after();
+        issue_pv(t, 1, false);
+        if (more) {
+          issue_qk(t + 1, natoms);
+          tc_commit(bar(B_SFULL + X));  // S(v + 1) is there, and every product before it is complete
+        } else {
+          tc_commit(bar(B_OFULL + X));
+        }
+        if (ATF_ORDER_BATCHES) {
+          const bool other_waits = X == 0 ? t + 1 < nB : (t >= 1 && t <= nA);
+          if (other_waits) mbar_arrive(bar(B_ORDER + X));
+        }
         tc_commit(bar(B_VEMPTY + t % VS));
       }
       for (int t = toff + nX; t < Tt && ok; ++t) ok = skip_v(t);
@@ -540,11 +560,11 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t e_next = v + 1 < nX ? __ldg(sched + 4 * (v + 1)) : 0u;
         const int ks = t % KS;
         bool handed_over = false;
+        if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 36; break; }
+        tc_fence_after();
 #pragma unroll 1
         for (int h = 0; h < 2; ++h) {
           const int c0 = h * HK;
-          if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 36; break; }
-          tc_fence_after();
           float s[HK];
           tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
           tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
@@ -570,10 +590,7 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             if (MODE == ATF_MODE_EXACT && v + 1 < nX) {
               const int p_keep = SchedEntry(e_next).p_mid;
-              if (p_keep < zeroed_from) {
-                if (!wait_or_abort(bar(B_SFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 37; break; }
-                zero_q_down_to(p_keep);
-              }
+              zero_q_down_to(p_keep);  // S(v) is complete, and S(v + 1) is not issued before both halves of P are signalled
             }
           }
           tc_wait_st();
@@ -609,11 +626,11 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
       }
 
+      if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
+      tc_fence_after();
 #pragma unroll 1
       for (int h = h_enter; h < 2; ++h) {
         const int c0 = h * HK;  // first key column of this half
-        if (!wait_or_abort(bar(B_SFULL + 2 * X + h), v & 1, abortp)) { ok = false; fail_site = 32; break; }
-        tc_fence_after();
         float s[HK];
         if (natoms > 0) {
           tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
@@ -711,11 +728,12 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             moved = !(v == 0 && h == 0);  // nothing has been accumulated before the first half
           }
           if (__any_sync(0xffffffffu, moved)) {  // rare after the first tiles
-            // every product issued so far must be complete: the issuer signals the other half's S
-            // barrier after each product (S(v, 1) follows P(v-1, 1) V; S(v+1, 0) follows P(v, 0) V)
-            const int vo = h == 0 ? v : v + 1;
-            if (!wait_or_abort(bar(B_SFULL + 2 * X + (h ^ 1)), vo & 1, abortp)) { ok = false; fail_site = 34; break; }
-            tc_fence_after();
+            // Every product into O issued so far must be complete.  Those of the earlier steps are:
+            // S(v) was issued after them.  In the second half, O += P(v, 0) V is on its way too.
+            if (h == 1) {
+              if (!wait_or_abort(bar(B_PV0 + X), v & 1, abortp)) { ok = false; fail_site = 34; break; }
+              tc_fence_after();
+            }
   #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {
               uint32_t o[32];
@@ -750,16 +768,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
               }
             }
           }
-          // Zero the Q columns that stop being live in most cells at the next step.  S(v + 1, 0) is
-          // issued once this half of P is signalled, so the zeroing has to happen here; S(v, 1) still
-          // needs the columns, so wait until it has been computed (it was issued long ago).
-          if (MODE == ATF_MODE_EXACT && v + 1 < nX) {
-            const int p_keep = SchedEntry(e_next).p_mid;
-            if (p_keep < zeroed_from) {
-              if (!wait_or_abort(bar(B_SFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 35; break; }
-              zero_q_down_to(p_keep);
-            }
-          }
+          // Zero the Q columns that stop being live in most cells at the next step: S(v) is complete,
+          // and S(v + 1) is not issued before both halves of P are signalled.
+          if (MODE == ATF_MODE_EXACT && v + 1 < nX) zero_q_down_to(SchedEntry(e_next).p_mid);
         }
         tc_wait_st();
         tc_fence_before();
