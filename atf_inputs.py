@@ -44,8 +44,8 @@ def qwen05b(N, outlier=False):
     return Workload("qwen2.5-0.5b", 1, 14, 2, 64, N, 1e6, 2.0, None, SEED0 + (3 if outlier else 2), outlier)
 
 
-def llama32_3b(N, B=1, seed_off=4):
-    return Workload("llama-3.2-3b", B, 24, 8, 128, N, 5e5, 2.0, LLAMA3_SCALING, SEED0 + seed_off)
+def llama32_3b(N, B=1, seed_off=4, outlier=False):
+    return Workload("llama-3.2-3b", B, 24, 8, 128, N, 5e5, 2.0, LLAMA3_SCALING, SEED0 + seed_off, outlier)
 
 
 def qwen7b_1m(N):

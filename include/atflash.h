@@ -38,7 +38,9 @@ enum {
   ATF_ERR_UNSUPPORTED = 2, /* valid request the library does not implement                   */
   ATF_ERR_CUDA = 3,        /* a CUDA runtime/driver call failed (text in atf_last_error)      */
   ATF_ERR_WORKSPACE = 4,   /* no workspace bound, or it is too small for this call            */
-  ATF_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out during an earlier launch     */
+  ATF_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out during an earlier launch; only
+                              atf_check_status / atf_check_status_at report it, and the results
+                              of that launch are not valid                                     */
 };
 
 /* Modes (second argument of the *_ex calls).
@@ -90,7 +92,8 @@ typedef struct {
  *   w_out[r] = floor(min(k * 2*pi/theta'_r, N)) for r in [0, d/2): the predicate "z <= w_r" on
  *   integer distances only sees the integer part.  k = INFINITY gives w_out[r] = N.
  *   theta_out (host, d/2 doubles) receives theta'_r if not NULL (the input atf_rope wants).
- * Errors: ATF_ERR_INVALID_ARG for d odd or <= 0, N < 1, k < 0 or NaN, null w_out.             */
+ * Errors: ATF_ERR_INVALID_ARG for d odd or <= 0, N < 1, k < 0 or NaN, null w_out, or llama3
+ *   scaling without factor > 0, 0 < low_freq_factor < high_freq_factor and original_ctx > 0.  */
 atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_scaling* s,
                             int64_t* w_out, double* theta_out);
 
@@ -146,10 +149,10 @@ atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, 
                           const atf_opts* opts, void* stream);
 
 /* Appended rows: the context already holds keys 0..N-Nq-1; the Nq new query rows sit at the
- * positions N-Nq..N-1 and attend to all N keys (App. C, "The interval itself": the row interval
- * [n0, n1] whose two endpoints are the whole prefill and the decode step; Sec. 7.3 runs the 1M
- * prefill as such chunks).  Every row gets exactly what atf_prefill gives it at that position
- * of a length-N prompt: a prefill cut into chunks is bit-identical to the single shot.
+ * positions N-Nq..N-1 and attend to all N keys.  This is the row interval [n0, n1] of App. C
+ * ("The interval itself"), whose two end points are the whole prefill and the decode step, and
+ * the chunked prefill of Sec. 7.3.  Every row gets exactly what atf_prefill gives it at that
+ * position of a length-N prompt, so a prefill cut into chunks has the bits of the single shot.
  *   Q, O: dev bf16 [B, Hq, Nq, d];  LSE: dev fp32 [B, Hq, Nq] or NULL;
  *   K, V: dev bf16 [B, Hkv, N, d], rotated at positions 0..N-1;  1 <= Nq <= N (else
  *   ATF_ERR_INVALID_ARG).  table, causal, opts, workspace, errors: as atf_prefill; the table's
@@ -172,8 +175,9 @@ atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, voi
  * pageable ones work but serialise.
  *   dev_scratch: device memory, 256-byte aligned, at least atf_prefill_host_scratch_bytes(...)
  *   bytes (the K/V caches, two Q / O / LSE chunk buffers and the prefill workspace; its first
- *   bytes are a workspace header: binding it with atf_bind_workspace lets atf_check_status read
- *   the kernels' status afterwards).  opts->workspace must be NULL.  The library allocates no
+ *   bytes are a workspace header, which the caller zero-fills once: atf_check_status_at, or
+ *   atf_check_status after binding it with atf_bind_workspace, reads the kernels' status
+ *   there).  opts->workspace must be NULL.  The library allocates no
  *   device memory; it creates two copy streams per device at the first call and keeps them.
  *   The call returns once everything is queued; `stream` (and the host results) are complete when
  *   the caller has synchronised `stream`.  Work already queued on `stream` is waited for.
@@ -189,7 +193,12 @@ atf_status atf_prefill_host(const void* Qh, const void* Kh, const void* Vh, void
  * so key m is at distance z = L-1-m.
  *   q, O: dev bf16 [B, Hq, d];  Kcache, Vcache: dev bf16 [B, Hkv, L, d] (the layout of K and V
  *   in atf_prefill, so a prefill cache is read with no conversion).
- *   Only the live low-frequency segments of each key row are read; V rows are read in full.
+ *   What is read: V rows in full.  K in this row layout: every row in full (a key no pair reaches
+ *   is skipped) with the dead pairs masked on chip - each 128-byte half of a row ends in live
+ *   low-frequency pairs and DRAM moves 128-byte lines, so leaving out the dead part of a row
+ *   saves no traffic.  The memory side of the window (Sec. 3.3) needs the tiled group-major K
+ *   cache (ATF_KLAYOUT_GROUPS through atf_decode_ex), in which only the live prefix of each tile
+ *   is fetched.
  *   Needs a workspace of atf_workspace_bytes(ATF_OP_DECODE, ...).                             */
 atf_status atf_decode(const void* q, const void* Kcache, const void* Vcache, void* O, int B,
                       int Hq, int Hkv, int64_t L, int d, const int64_t* table, void* stream);
@@ -197,8 +206,8 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
                          int Hq, int Hkv, int64_t L, int d, const int64_t* table,
                          const atf_opts* opts, void* stream);
 
-/* Copies n rotated key rows into a group-major K cache (see ATF_KLAYOUT_GROUPS; Sec. 3.3's
- * "out-of-window components are not loaded" made to hold at DRAM line granularity).
+/* Copies n rotated key rows into a group-major K cache (see ATF_KLAYOUT_GROUPS: the layout in
+ * which the memory side of the window, Sec. 3.3, holds at DRAM line granularity).
  *   K : dev bf16 [B, Hkv, n, d], rows for positions pos0 .. pos0+n-1;
  *   Kg: dev bf16 [B, Hkv, ceil(Lcap/KT), d/16, KT, 16], the cache, Lcap >= pos0 + n its length
  *       in keys, KT = atf_kcache_tile_keys(d) (64 for d = 128, 128 for d = 64).
@@ -231,7 +240,9 @@ atf_status atf_decode_static(const void* q, const void* Kcache, const void* Vcac
 
 /* Workspace.  The library keeps no allocation of its own: the caller allocates
  * atf_workspace_bytes() bytes of device memory (256-byte aligned), zero-fills it once, and
- * binds it (per process; the pointer is only stored).  A workspace sized for the largest call
+ * binds it.  The binding is ONE pointer per process (it is only stored), not one per device: a
+ * process that drives several GPUs passes each call its own workspace in atf_opts.workspace.
+ * A workspace sized for the largest call
  * serves prefill and decode in turn: its first 64.25 KiB (status words and decode's split
  * counters, which the kernels leave zeroed) are never used as scratch.  One call at a time may use a given
  * workspace; calls that overlap on the GPU need separate workspaces (atf_opts.workspace).     */
@@ -239,9 +250,19 @@ enum { ATF_OP_PREFILL = 0, ATF_OP_DECODE = 1 };
 size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d);
 atf_status atf_bind_workspace(void* dev_ptr, size_t bytes);
 
-/* Reads (and clears) the device status word of the bound workspace; synchronises `stream`.
- * Returns ATF_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last check.        */
+/* Reads (and clears) the device status words of the bound workspace and, if atf_decode_static
+ * has run on the current device, of its built-in array; synchronises `stream`.  Returns
+ * ATF_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last check (every device-side
+ * wait gives up after 2 s of wall time and the kernel then ends; its results are not valid).
+ * atf_check_status_at does the same for a workspace that was passed in atf_opts.workspace or as
+ * dev_scratch of atf_prefill_host (which leaves the status words of earlier calls in place).   */
 atf_status atf_check_status(void* stream);
+atf_status atf_check_status_at(void* workspace, void* stream);
+
+/* Self-test of that report path: launches one small kernel that waits, with the kernels' bounded
+ * wait and a limit of limit_us microseconds (1..100000), for a barrier nobody signals, gives up
+ * and records it in the bound workspace.  The next atf_check_status returns ATF_ERR_TIMEOUT once. */
+atf_status atf_selftest_bounded_wait(unsigned int limit_us, void* stream);
 
 /* Text of the calling thread's last error ("" if none). Never NULL. */
 const char* atf_last_error(void);

@@ -68,6 +68,8 @@ def effective_theta(base: float, d: int, scaling: dict | None = None) -> np.ndar
     lf = float(scaling["low_freq_factor"])
     hf = float(scaling["high_freq_factor"])
     c = float(scaling["original_ctx"])
+    if not (f > 0.0 and 0.0 < lf < hf and c > 0.0 and math.isfinite(f) and math.isfinite(hf)):
+        raise ValueError("llama3 scaling needs factor > 0, 0 < low_freq_factor < high_freq_factor, original_ctx > 0")
     out = np.empty_like(theta)
     for r in range(h):
         lam = 2.0 * math.pi / theta[r]

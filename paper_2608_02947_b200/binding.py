@@ -73,11 +73,13 @@ def lib():
     L.atf_workspace_bytes.restype = C.c_size_t
     L.atf_bind_workspace.argtypes = [vp, C.c_size_t]
     L.atf_check_status.argtypes = [vp]
+    L.atf_check_status_at.argtypes = [vp, vp]
+    L.atf_selftest_bounded_wait.argtypes = [C.c_uint, vp]
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
                  "atf_kcache_pack",
-                 "atf_bind_workspace", "atf_check_status"):
+                 "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -134,6 +136,15 @@ def _stream(t):
     return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
 
 
+def _one_device(*tensors):
+    """All device tensors of a call must live on one GPU: the C side launches on the current device, and the
+    binding makes that the tensors' device for the duration of the call."""
+    devs = {t.device for t in tensors if t is not None}
+    if len(devs) != 1:
+        raise AtfError(1, f"all tensors of a call must be on the same CUDA device (got {sorted(map(str, devs))})")
+    return torch.cuda.device(devs.pop())
+
+
 def _dev_bf16(t, name):
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
         raise AtfError(1, f"{name} must be a contiguous CUDA bf16 tensor")
@@ -181,7 +192,8 @@ def atf_rope(X, theta, pos0=0):
     B, H, N, d = X.shape
     th = torch.as_tensor(theta, dtype=torch.float64).cpu()
     arr = (C.c_double * th.numel())(*th.tolist())
-    _check(lib().atf_rope(C.c_void_p(X.data_ptr()), B, H, N, d, arr, int(pos0), _stream(X)))
+    with torch.cuda.device(X.device):
+        _check(lib().atf_rope(C.c_void_p(X.data_ptr()), B, H, N, d, arr, int(pos0), _stream(X)))
     return X
 
 
@@ -244,19 +256,21 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
         O = torch.empty_like(Q)
     if LSE is None and return_lse:
         LSE = torch.empty((B, Hq, Nq), dtype=torch.float32, device=Q.device)
+    dev = _one_device(Q, K, V, O, LSE, kept_terms)
     ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL, B, Hq, Hkv, N, d), Q.device)
     tab, _keep = _table_ptr(table, d)
     o = _opts(mode, kept_terms, None)
     lse_ptr = C.c_void_p(LSE.data_ptr()) if LSE is not None else None
-    if Nq == N:
-        _check(lib().atf_prefill_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
-                                    C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv, N, d, tab, 1 if causal else 0,
-                                    C.byref(o) if o is not None else None, _stream(Q)))
-    else:
-        _check(lib().atf_prefill_chunk_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()),
-                                          C.c_void_p(V.data_ptr()), C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv,
-                                          Nq, N, d, tab, 1 if causal else 0,
-                                          C.byref(o) if o is not None else None, _stream(Q)))
+    with dev:
+        if Nq == N:
+            _check(lib().atf_prefill_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                        C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+                                        C.byref(o) if o is not None else None, _stream(Q)))
+        else:
+            _check(lib().atf_prefill_chunk_ex(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()),
+                                              C.c_void_p(V.data_ptr()), C.c_void_p(O.data_ptr()), lse_ptr, B, Hq, Hkv,
+                                              Nq, N, d, tab, 1 if causal else 0,
+                                              C.byref(o) if o is not None else None, _stream(Q)))
     if on_host:
         return _to_pinned_host(O, O_host), (_to_pinned_host(LSE, LSE_host) if LSE is not None else None)
     return O, LSE
@@ -312,8 +326,9 @@ def atf_kcache_pack(K, Kg=None, pos0=0):
     _dev_bf16(Kg, "Kg")
     if Kg.dim() != 6 or Kg.shape[:2] != (B, Hkv) or Kg.shape[3:] != (d // 16, kt, 16):
         raise AtfError(1, f"Kg must be [B,Hkv,tiles,d/16,{kt},16]")
-    _check(lib().atf_kcache_pack(C.c_void_p(K.data_ptr()), C.c_void_p(Kg.data_ptr()), B, Hkv, n, Kg.shape[2] * kt,
-                                 int(pos0), d, _stream(K)))
+    with _one_device(K, Kg):
+        _check(lib().atf_kcache_pack(C.c_void_p(K.data_ptr()), C.c_void_p(Kg.data_ptr()), B, Hkv, n, Kg.shape[2] * kt,
+                                     int(pos0), d, _stream(K)))
     return Kg
 
 
@@ -338,12 +353,14 @@ def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=No
     if O is None:
         O = torch.empty_like(q)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
+    dev = _one_device(q, Kcache, Vcache, O, kept_terms)
     ensure_workspace(atf_workspace_bytes(ATF_OP_DECODE, B, Hq, Hkv, L, d), q.device)
     tab, _keep = _table_ptr(table, d)
     o = _opts(mode, kept_terms, lse, k_layout)
-    _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
-                               C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,
-                               C.byref(o) if o is not None else None, _stream(q)))
+    with dev:
+        _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
+                                   C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,
+                                   C.byref(o) if o is not None else None, _stream(q)))
     if on_host:
         return (_to_pinned_host(O), _to_pinned_host(lse)) if return_lse else _to_pinned_host(O)
     return (O, lse) if return_lse else O
@@ -355,15 +372,36 @@ def atf_decode_static(q, Kcache, Vcache, table=None, O=None):
     Only argument marshalling happens here; pass O to avoid the one output allocation."""
     for t, nm in ((q, "q"), (Kcache, "Kcache"), (Vcache, "Vcache")):
         _dev_bf16(t, nm)
+    if q.dim() != 3 or Kcache.dim() != 4:
+        raise AtfError(1, "q must be [B,Hq,d] and Kcache [B,Hkv,L,d]")
     B, Hq, d = q.shape
     Hkv, L = Kcache.shape[1], Kcache.shape[2]
+    if tuple(Kcache.shape) != (B, Hkv, L, d) or Vcache.shape != Kcache.shape:
+        raise AtfError(1, "Kcache and Vcache must both be [B,Hkv,L,d], matching q [B,Hq,d]")
     if O is None:
         O = torch.empty_like(q)
+    if O.shape != q.shape:
+        raise AtfError(1, "O must have the shape of q")
+    _dev_bf16(O, "O")
     tab, _keep = _table_ptr(table, d)
-    _check(lib().atf_decode_static(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
-                                   C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab, _stream(q)))
+    with _one_device(q, Kcache, Vcache, O):
+        _check(lib().atf_decode_static(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()),
+                                       C.c_void_p(Vcache.data_ptr()), C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,
+                                       _stream(q)))
     return O
 
 
-def check_status():
-    _check(lib().atf_check_status(C.c_void_p(torch.cuda.current_stream().cuda_stream)))
+def check_status(workspace=None):
+    """Raises AtfError(ATF_ERR_TIMEOUT) if a kernel gave up a bounded wait since the last check: in the bound
+    workspace (and the built-in array of atf_decode_static), or in the given workspace tensor."""
+    if workspace is None:
+        _check(lib().atf_check_status(C.c_void_p(torch.cuda.current_stream().cuda_stream)))
+    else:
+        with torch.cuda.device(workspace.device):
+            _check(lib().atf_check_status_at(C.c_void_p(workspace.data_ptr()),
+                                             C.c_void_p(torch.cuda.current_stream(workspace.device).cuda_stream)))
+
+
+def selftest_bounded_wait(limit_us=1000):
+    """Launches the library's wait-that-runs-out self-test on the current device (needs a bound workspace)."""
+    _check(lib().atf_selftest_bounded_wait(int(limit_us), C.c_void_p(torch.cuda.current_stream().cuda_stream)))

@@ -39,6 +39,8 @@ struct AtfWorkspace {
   size_t bytes;
 };
 AtfWorkspace atf_bound_workspace();
+// atf_check_status also reads (and clears) the status words registered here for the device
+void atf_register_status_words(int device, void* dev_ptr);
 
 // decode CTAs resident on the GPU at once: 2 per SM when K is read in the row layout, 3 per SM
 // with the group-major K cache (measured: whole-row streaming is fastest with fewer blocks in

@@ -1,13 +1,19 @@
 // atf_decode: split-K windowed attention of one query row per (batch, head) against a
-// contiguous KV cache (Sec. 5; the last row of Fig. 3).  Bandwidth-bound: the cache is moved
-// with 16-byte asynchronous copies, a row of the cache is covered by consecutive lanes, and a
-// 16-byte chunk of a key row that lies wholly outside the key's live pair range is not read
-// (Sec. 3.3: out-of-window components are not brought on chip) - its place in shared memory is
-// zero-filled instead.  V rows are read in full.
+// contiguous KV cache (Sec. 5; the last row of Fig. 3).  Bandwidth-bound: what matters is which
+// bytes leave DRAM.
 //
-// Work split: grid = (splits, Hkv, B).  A block owns a contiguous key range and each of its 4
-// warps walks that range in blocks of 2048/d keys through its own 3-stage cp.async ring.  Per
-// block a warp computes, for the (up to 8) query heads that share the KV head at once:
+// K cache layouts.  In the row layout [L, d] (the layout atf_prefill takes) every 128-byte half
+// of a key row ends in live low-frequency pairs, and DRAM moves whole 128-byte lines, so the
+// window cannot save traffic there: rows are copied whole and the dead pairs are masked in
+// registers (a key no pair reaches is not copied at all).  In the tiled group-major layout
+// (written by atf_kcache_pack or by atf_prefill itself) the pairs a far key keeps are a contiguous
+// prefix of each tile, and only that prefix is fetched (Sec. 3.3: components outside the window
+// never come on chip).  V rows are read in full in both.
+//
+// Work split: grid = (splits, Hkv, B).  Tiles of 64 (d = 128) or 128 (d = 64) keys are dealt
+// round-robin to the splits; each of a block's 4 warps takes a quarter of a tile through its own
+// two-stage cp.async ring.  Per block of keys a warp computes, for the (up to 8) query heads that
+// share the KV head at once:
 //   S = q K^T   with mma.sync (m16n8k16, bf16 in, fp32 accumulate; the heads are the M rows),
 //   the online softmax in registers (log2 domain, lazy rescaling),
 //   O += P V    with mma.sync, V fragments transposed by ldmatrix.
@@ -679,6 +685,7 @@ extern "C" atf_status atf_decode_static(const void* q, const void* Kcache, const
                                         int Hkv, int64_t L, int d, const int64_t* table, void* stream) {
   if (B < 1 || Hq < 1 || Hkv < 1 || L < 1 || (d != 64 && d != 128) || Hq % Hkv)
     return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode_static: bad shape");
+  if ((int64_t)B * Hkv > ATF_WS_COUNTER_SLOTS) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode_static: B*Hkv must be <= %d", ATF_WS_COUNTER_SLOTS);
   const size_t need = decode_ws_bytes(B, Hq, Hkv, L, d);
   if (need > ATF_STATIC_SCRATCH_BYTES)
     return atf_fail(ATF_ERR_WORKSPACE,
@@ -693,12 +700,15 @@ extern "C" atf_status atf_decode_static(const void* q, const void* Kcache, const
     ATF_CUDA_CHECK(cudaGetSymbolAddress(&p, g_atf_static_scratch));
     if (!p) return atf_fail(ATF_ERR_CUDA, "atf_decode_static: cudaGetSymbolAddress returned a null address");
     g_static_scratch_ptr[dev] = p;
+    atf_register_status_words(dev, p);
   }
   void* scratch = g_static_scratch_ptr[dev];
-  // The array keeps whatever the last call left: the status words and the split counters must
-  // start at zero (a memset on the stream, not an allocation); the partials are overwritten.
-  const size_t clear = ATF_WS_STATUS_BYTES + (size_t)B * Hkv * sizeof(unsigned int);
-  ATF_CUDA_CHECK(cudaMemsetAsync(scratch, 0, clear, (cudaStream_t)stream));
+  // The array keeps whatever the last call left.  The split counters must start at zero (the kernel
+  // leaves them so, but a launch that gave up may not have): a memset on the stream, not an
+  // allocation.  The partials are overwritten; the status words are left alone, so that a give-up of
+  // an earlier launch is still there for atf_check_status.
+  ATF_CUDA_CHECK(cudaMemsetAsync((char*)scratch + ATF_WS_STATUS_BYTES, 0, (size_t)B * Hkv * sizeof(unsigned int),
+                                 (cudaStream_t)stream));
   atf_opts o;
   memset(&o, 0, sizeof(o));
   o.mode = ATF_MODE_EXACT;

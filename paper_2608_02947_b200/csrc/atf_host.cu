@@ -4,11 +4,18 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <initializer_list>
 
 #include "atf_common.cuh"
 
 static thread_local char g_err[512] = "";
 static AtfWorkspace g_ws = {nullptr, 0};
+// further places a kernel may have left a status in: the built-in scratch of atf_decode_static, per device
+static void* g_extra_status[64] = {nullptr};
+
+void atf_register_status_words(int device, void* dev_ptr) {
+  if (device >= 0 && device < 64) g_extra_status[device] = dev_ptr;
+}
 
 atf_status atf_fail(atf_status code, const char* fmt, ...) {
   va_list ap;
@@ -59,6 +66,27 @@ atf_status atf_validate_table(const char* who, const int64_t* table, int d, int6
   return ATF_OK;
 }
 
+// Waits on a barrier nobody arrives on, with the kernels' own bounded wait but a short limit, and
+// reports the give-up the way they do (status word 0 = 1, word 1 = the site).
+__global__ void atf_bounded_wait_selftest_kernel(unsigned int* status, unsigned long long limit_ns) {
+  __shared__ alignas(8) unsigned long long barmem;
+  const uint32_t bar = smem_u32(&barmem);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    mbar_fence_init();
+    bool done = mbar_try_wait(bar, 0);
+    const unsigned long long t0 = global_timer_ns();
+    while (!done && global_timer_ns() - t0 <= limit_ns) {
+#pragma unroll 1
+      for (int i = 0; i < 64 && !done; ++i) done = mbar_try_wait(bar, 0);
+    }
+    if (!done) {
+      atomicExch(status, 1u);
+      atomicExch(status + 1, 99u);
+    }
+  }
+}
+
 size_t atf_decode_workspace_bytes(int B, int Hq, int Hkv, int64_t L, int d);
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d);
 
@@ -81,6 +109,11 @@ atf_status atf_window_table(double base, int d, double k, int64_t N, const atf_s
   if (!(base > 1.0)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: base must be > 1");
   if (!w_out) return atf_fail(ATF_ERR_INVALID_ARG, "atf_window_table: w_out is NULL");
   if (s && s->kind != 0 && s->kind != 1) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_window_table: unknown scaling kind %d", s->kind);
+  if (s && s->kind == 1 &&
+      !(s->factor > 0.0 && s->low_freq_factor > 0.0 && s->high_freq_factor > s->low_freq_factor && s->original_ctx > 0 &&
+        s->factor < INFINITY && s->high_freq_factor < INFINITY))
+    return atf_fail(ATF_ERR_INVALID_ARG,
+                    "atf_window_table: llama3 scaling needs factor > 0, 0 < low_freq_factor < high_freq_factor and original_ctx > 0");
   const double two_pi = 2.0 * M_PI;
   const int h = d / 2;
   for (int r = 0; r < h; ++r) {
@@ -158,17 +191,50 @@ atf_status atf_bind_workspace(void* dev_ptr, size_t bytes) {
   return ATF_OK;
 }
 
-atf_status atf_check_status(void* stream) {
-  if (!g_ws.ptr) return atf_fail(ATF_ERR_WORKSPACE, "atf_check_status: no workspace bound");
-  unsigned int st[2] = {0, 0};
-  cudaStream_t s = (cudaStream_t)stream;
-  ATF_CUDA_CHECK(cudaMemcpyAsync(st, g_ws.ptr, sizeof(st), cudaMemcpyDeviceToHost, s));
+// Reads and clears two status words at `words` (device); *hit receives whether a kernel had given up.
+static atf_status read_status_words(void* words, cudaStream_t s, unsigned int* st) {
+  st[0] = st[1] = 0;
+  ATF_CUDA_CHECK(cudaMemcpyAsync(st, words, 2 * sizeof(unsigned int), cudaMemcpyDeviceToHost, s));
   ATF_CUDA_CHECK(cudaStreamSynchronize(s));
   if (st[0] != 0) {
-    ATF_CUDA_CHECK(cudaMemsetAsync(g_ws.ptr, 0, sizeof(st), s));
+    ATF_CUDA_CHECK(cudaMemsetAsync(words, 0, 2 * sizeof(unsigned int), s));
     ATF_CUDA_CHECK(cudaStreamSynchronize(s));
-    return atf_fail(ATF_ERR_TIMEOUT, "a kernel gave up a bounded wait (code %u at site %u)", st[0], st[1]);
   }
+  return ATF_OK;
+}
+
+atf_status atf_check_status_at(void* workspace, void* stream) {
+  if (!workspace) return atf_fail(ATF_ERR_INVALID_ARG, "atf_check_status_at: workspace is NULL");
+  unsigned int st[2];
+  atf_status rc = read_status_words(workspace, (cudaStream_t)stream, st);
+  if (rc != ATF_OK) return rc;
+  if (st[0] != 0) return atf_fail(ATF_ERR_TIMEOUT, "a kernel gave up a bounded wait (code %u at site %u)", st[0], st[1]);
+  return ATF_OK;
+}
+
+atf_status atf_selftest_bounded_wait(unsigned int limit_us, void* stream) {
+  if (!g_ws.ptr) return atf_fail(ATF_ERR_WORKSPACE, "atf_selftest_bounded_wait: no workspace bound");
+  if (limit_us < 1 || limit_us > 100000) return atf_fail(ATF_ERR_INVALID_ARG, "atf_selftest_bounded_wait: limit must be 1..100000 us");
+  atf_bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((unsigned int*)g_ws.ptr, 1000ull * limit_us);
+  ATF_CUDA_CHECK(cudaGetLastError());
+  return ATF_OK;
+}
+
+atf_status atf_check_status(void* stream) {
+  int dev = -1;
+  void* extra = (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) ? g_extra_status[dev] : nullptr;
+  if (!g_ws.ptr && !extra) return atf_fail(ATF_ERR_WORKSPACE, "atf_check_status: no workspace bound");
+  unsigned int st[2] = {0, 0}, hit[2] = {0, 0};
+  for (void* words : {g_ws.ptr, extra}) {
+    if (!words) continue;
+    atf_status rc = read_status_words(words, (cudaStream_t)stream, st);
+    if (rc != ATF_OK) return rc;
+    if (st[0] != 0 && hit[0] == 0) {
+      hit[0] = st[0];
+      hit[1] = st[1];
+    }
+  }
+  if (hit[0] != 0) return atf_fail(ATF_ERR_TIMEOUT, "a kernel gave up a bounded wait (code %u at site %u)", hit[0], hit[1]);
   return ATF_OK;
 }
 

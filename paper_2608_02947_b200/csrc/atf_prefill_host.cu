@@ -125,7 +125,9 @@ extern "C" atf_status atf_prefill_host(const void* Qh, const void* Kh, const voi
     HOST_CHECK(cudaEventCreateWithFlags(&out_done[c], cudaEventDisableTiming));
   }
   // everything follows the work already queued on the caller's stream
-  HOST_CHECK(cudaMemsetAsync(ws, 0, ATF_WS_HEADER, comp));
+  // the split counters start at zero; the status words are left as they are (the caller zero-fills the
+  // header once), so a give-up of an earlier call is still there for atf_check_status
+  HOST_CHECK(cudaMemsetAsync(ws + ATF_WS_STATUS_BYTES, 0, ATF_WS_HEADER - ATF_WS_STATUS_BYTES, comp));
   HOST_CHECK(cudaEventRecord(start_ev, comp));
   HOST_CHECK(cudaStreamWaitEvent(st->h2d, start_ev, 0));
   HOST_CHECK(cudaStreamWaitEvent(st->d2h, start_ev, 0));

@@ -72,6 +72,42 @@ def test_validation_returns_codes_without_a_device(atf):
     assert lib.atf_kcache_tile_keys(128) == 64 and lib.atf_kcache_tile_keys(64) == 128
 
 
+def test_degenerate_scaling_is_refused_by_both_sides(atf):
+    """A llama3 scaling whose blend is undefined (equal factors, non-positive factor or context) would give an
+    infinite or NaN frequency: the C side answers ATF_ERR_INVALID_ARG, the oracle raises."""
+    for bad in (dict(high_freq_factor=1.0), dict(factor=0.0), dict(factor=-2.0), dict(original_ctx=0),
+                dict(low_freq_factor=0.0), dict(low_freq_factor=5.0), dict(factor=math.inf)):
+        sc = dict(LLAMA3_SCALING, **bad)
+        with pytest.raises(atf.AtfError) as e:
+            atf.atf_window_table(5e5, 128, 2.0, 8192, sc)
+        assert e.value.code == 1
+        with pytest.raises(ValueError):
+            orc.window_table(5e5, 128, 2.0, 8192, sc)
+        with pytest.raises(atf.AtfError):
+            atf.atf_window_table_family(5e5, 128, 8192, sc)
+
+
+def test_static_decode_and_status_refusals_without_a_device(atf):
+    lib = atf.lib()
+    fake = C.c_void_p(4096)
+    # shapes are checked before anything touches a device
+    assert lib.atf_decode_static(fake, fake, fake, fake, 0, 24, 8, 1024, 128, None, None) == 1
+    assert lib.atf_decode_static(fake, fake, fake, fake, 1, 24, 7, 1024, 128, None, None) == 1
+    assert lib.atf_decode_static(fake, fake, fake, fake, 1, 24, 8, 1024, 96, None, None) == 1
+    # a problem beyond the built-in array is refused with both sizes in the text
+    assert lib.atf_decode_static(fake, fake, fake, fake, 64, 24, 8, 131072, 128, None, None) == 4
+    msg = lib.atf_last_error().decode()
+    assert str(lib.atf_decode_static_capacity()) in msg and "atf_decode" in msg
+    assert lib.atf_check_status_at(None, None) == 1
+    assert lib.atf_selftest_bounded_wait(0, None) in (1, 4)   # no workspace bound, or a limit out of range
+    # the binding refuses tensors that are not CUDA bf16, and a cache that does not match q, before the C call
+    import torch
+    q = torch.zeros((1, 24, 128), dtype=torch.bfloat16)
+    kc = torch.zeros((1, 8, 64, 128), dtype=torch.bfloat16)
+    with pytest.raises(atf.AtfError):
+        atf.atf_decode_static(q, kc, kc)
+
+
 FAMILY_CASES = [
     dict(),  # Eq. 3 with k = 2
     dict(k_hi=64.0),

@@ -11,6 +11,18 @@ from oracle import atf_oracle as orc
 
 pytestmark = pytest.mark.gpu
 O_MAX, O_MEAN, LSE_TOL = 2e-2, 2e-3, 1e-3
+# With i.i.d. inputs a late row's output is small (an average over many keys), so the absolute
+# tolerances alone say little there: each sampled row must also agree with the oracle to a few percent
+# of that row's own magnitude (bf16 rounding of P and of O gives a few tenths of a percent).
+ROW_REL = 0.05
+
+
+def _check_rows(O_gpu_rows, O_ref, tag):
+    err = np.abs(O_gpu_rows - O_ref)
+    assert np.isfinite(O_gpu_rows).all(), tag
+    assert err.max() <= O_MAX and err.mean() <= O_MEAN, (tag, err.max(), err.mean())
+    rel = np.sqrt((err ** 2).sum(axis=-1)) / np.maximum(np.sqrt((O_ref ** 2).sum(axis=-1)), 1e-30)
+    assert rel.max() <= ROW_REL, (tag, float(rel.max()), int(rel.argmax()))
 
 
 @pytest.fixture(scope="module")
@@ -51,9 +63,7 @@ def _prefill_fullsize(atf, w, heads, n_random, mode=0, tile_rows=True):
     g = w.Hq // w.Hkv
     for hq in heads:
         Or, Lr = _oracle_rows(Q[0, hq], K[0, hq // g], V[0, hq // g], theta_o, Wo, rows, mode, atf)
-        err = np.abs(gen.to_f64(O[0, hq][rows]) - Or)
-        assert np.isfinite(err).all()
-        assert err.max() <= O_MAX and err.mean() <= O_MEAN, (hq, err.max(), err.mean())
+        _check_rows(gen.to_f64(O[0, hq][rows]), Or, hq)
         assert np.abs(LSE[0, hq][rows].double().cpu().numpy() - Lr).max() <= LSE_TOL
 
 
@@ -73,6 +83,12 @@ def test_llama_8192(atf):
 
 def test_llama_32768(atf):
     _prefill_fullsize(atf, gen.llama32_3b(32768, seed_off=5), heads=[5], n_random=48, tile_rows=False)
+
+
+def test_llama_32768_outlier_channels(atf):
+    """Peaked scores (|s| up to ~100, outputs of order 1): a mishandled cell shows at full size, and rows whose
+    later scores overshoot the reference maximum of their first tile by far exercise the redo path."""
+    _prefill_fullsize(atf, gen.llama32_3b(32768, seed_off=13, outlier=True), heads=[2, 20], n_random=48, tile_rows=False)
 
 
 def test_llama_131072(atf):
@@ -143,6 +159,5 @@ def test_qwen7b_1m_prefill_counts_and_rows(atf):
         qn = orc.rope_half_split(qsel[i:i + 1], theta_o, pos0=n)[0]
         s = orc.windowed_scores_row(qn, Kr, Wo, n)
         o, l = orc._softmax_row(s, Vr[: n + 1])
-        err = np.abs(gen.to_f64(O[0, hq, n]) - o)
-        assert err.max() <= O_MAX and err.mean() <= O_MEAN, (n, err.max())
+        _check_rows(gen.to_f64(O[0, hq, n])[None, :], o[None, :], n)
         assert abs(float(LSE[0, hq, n]) - l) <= LSE_TOL
