@@ -65,14 +65,16 @@ typedef struct {
 
 /* Layout of the K cache handed to atf_decode_ex.
  * ATF_KLAYOUT_ROWS  : [B, Hkv, L, d], the layout of K in atf_prefill (default).
- * ATF_KLAYOUT_GROUPS: [B, Hkv, T, d/16, KT, 16] as written by atf_kcache_pack: the keys are cut
- *   into T = ceil(L/KT) tiles of KT = atf_kcache_tile_keys(d) keys (16 KiB per tile); inside a
- *   tile, group j holds, for each of its keys, the 8 pairs r = d/2-1-8j ... d/2-8-8j (lowest
- *   frequency first), each pair as (dim r, dim r + d/2) side by side.  The pairs a far key
- *   keeps (a low-frequency slice, Sec. 3.3) are then the leading groups, i.e. a contiguous
- *   prefix of the tile, so decode fetches only live bytes; in the row layout DRAM's 128-byte
- *   lines make it fetch every row whole.  This layout is an extension: the paper's ports keep
- *   the row layout.                                                                          */
+ * ATF_KLAYOUT_GROUPS: [B, Hkv, T, d/16, KT, 16] as written by atf_kcache_pack or by a prefill with
+ *   atf_opts.kcache_groups: the keys are cut into T = ceil(L/KT) tiles of KT =
+ *   atf_kcache_tile_keys(d) keys (16 KiB per tile); inside a tile, group j holds, for each of its
+ *   keys, the 8 pairs r = d/2-1-8j ... d/2-8-8j (lowest frequency first), each pair as (dim r,
+ *   dim r + d/2) side by side; for keys whose index in the tile has bit 2 set the two 16-byte
+ *   halves of that 32-byte entry are swapped (the copied image is then free of shared-memory
+ *   bank conflicts).  The pairs a far key keeps (a low-frequency slice, Sec. 3.3) are the
+ *   leading groups, i.e. a contiguous prefix of the tile, so decode fetches only live bytes, with
+ *   one bulk copy per tile; in the row layout DRAM's 128-byte lines make it fetch every row
+ *   whole.  This layout is an extension: the paper's ports keep the row layout.             */
 enum { ATF_KLAYOUT_ROWS = 0, ATF_KLAYOUT_GROUPS = 1 };
 
 /* Optional arguments of the *_ex calls.  Zero-initialise, then set what is needed. */
@@ -85,6 +87,13 @@ typedef struct {
   void* workspace;       /* dev scratch for this call, or NULL to use the bound workspace       */
   size_t workspace_bytes;
   int k_layout;          /* decode only: ATF_KLAYOUT_ROWS (default) or ATF_KLAYOUT_GROUPS        */
+  void* kcache_groups;   /* prefill only: dev, a group-major K cache (ATF_KLAYOUT_GROUPS) of
+                            kcache_capacity keys per (batch, KV head), or NULL.  If set, the prefill
+                            also writes the K rows of this call's new positions (N-Nq .. N-1; all
+                            of them for atf_prefill) into it, so that decode can read the cache
+                            the prefill wrote with no conversion pass (Sec. 7.2).               */
+  int64_t kcache_capacity; /* keys the group-major cache is laid out for, >= N (its tile count fixes the
+                              layout).  Decode with ATF_KLAYOUT_GROUPS reads it too: 0 = exactly L.    */
 } atf_opts;
 
 /* Window table (Eq. 2, Eq. 3; effective frequencies per Sec. 3.2).  Host only, no GPU needed.
@@ -211,7 +220,8 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
  *   K : dev bf16 [B, Hkv, n, d], rows for positions pos0 .. pos0+n-1;
  *   Kg: dev bf16 [B, Hkv, ceil(Lcap/KT), d/16, KT, 16], the cache, Lcap >= pos0 + n its length
  *       in keys, KT = atf_kcache_tile_keys(d) (64 for d = 128, 128 for d = 64).
- * atf_decode_ex with k_layout = ATF_KLAYOUT_GROUPS then wants ceil(L/KT) == ceil(Lcap/KT).    */
+ * atf_decode_ex with k_layout = ATF_KLAYOUT_GROUPS takes the cache with atf_opts.kcache_capacity = Lcap
+ * (0 means a cache of exactly ceil(L/KT) tiles).                                                */
 int64_t atf_kcache_tile_keys(int d);
 atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, int64_t n, int64_t Lcap,
                            int64_t pos0, int d, void* stream);

@@ -23,4 +23,5 @@ from .binding import (  # noqa: F401
     lib,
     lib_path,
     llama3_scaling,
+    new_kcache_groups,
 )

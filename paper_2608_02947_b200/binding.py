@@ -26,7 +26,8 @@ class _Scaling(C.Structure):
 
 class _Opts(C.Structure):
     _fields_ = [("mode", C.c_int), ("kept_terms", C.c_void_p), ("lse", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("k_layout", C.c_int)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("k_layout", C.c_int),
+                ("kcache_groups", C.c_void_p), ("kcache_capacity", C.c_int64)]
 
 
 def lib_path():
@@ -197,10 +198,13 @@ def atf_rope(X, theta, pos0=0):
     return X
 
 
-def _opts(mode, kept_terms, lse, k_layout=ATF_KLAYOUT_ROWS):
-    if mode == ATF_MODE_EXACT and kept_terms is None and lse is None and k_layout == ATF_KLAYOUT_ROWS:
+def _opts(mode, kept_terms, lse, k_layout=ATF_KLAYOUT_ROWS, kcache_groups=None):
+    if mode == ATF_MODE_EXACT and kept_terms is None and lse is None and k_layout == ATF_KLAYOUT_ROWS and kcache_groups is None:
         return None
     o = _Opts()
+    if kcache_groups is not None:
+        o.kcache_groups = kcache_groups.data_ptr()
+        o.kcache_capacity = kcache_groups.shape[2] * kcache_groups.shape[4]
     o.mode = int(mode)
     o.k_layout = int(k_layout)
     o.kept_terms = kept_terms.data_ptr() if kept_terms is not None else None
@@ -228,8 +232,21 @@ def _host_roundtrip(tensors):
     return [t.pin_memory().to("cuda", non_blocking=True) if not t.is_cuda else t for t in tensors]
 
 
+def new_kcache_groups(B, Hkv, capacity, d, device):
+    """A zeroed tiled group-major K cache for `capacity` keys per (batch, KV head): [B,Hkv,tiles,d/16,KT,16]."""
+    kt = int(lib().atf_kcache_tile_keys(d))
+    return torch.zeros((B, Hkv, (capacity + kt - 1) // kt, d // 16, kt, 16), dtype=torch.bfloat16, device=device)
+
+
+def _check_kcache_groups(Kg, B, Hkv, N, d):
+    kt = int(lib().atf_kcache_tile_keys(d))
+    _dev_bf16(Kg, "kcache_groups")
+    if Kg.dim() != 6 or Kg.shape[:2] != (B, Hkv) or Kg.shape[3:] != (d // 16, kt, 16) or Kg.shape[2] * kt < N:
+        raise AtfError(1, f"kcache_groups must be [B,Hkv,tiles,d/16,{kt},16] with room for N keys")
+
+
 def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
-                O=None, LSE=None):
+                O=None, LSE=None, kcache_groups=None):
     """Windowed causal attention.  Q [B,Hq,Nq,d], K/V [B,Hkv,N,d] bf16, already rotated.
 
     Nq == N is the whole prefill (atf_prefill_ex); Nq < N are appended rows: Q holds the last Nq
@@ -242,7 +259,7 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
     O_host = LSE_host = None
     if on_host and Q.shape[2] == K.shape[2]:
         return atf_prefill_host(Q, K, V, table=table, causal=causal, mode=mode, kept_terms=kept_terms,
-                                return_lse=return_lse, O=O, LSE=LSE)
+                                return_lse=return_lse, O=O, LSE=LSE, kcache_groups=kcache_groups)
     if on_host:
         Q, K, V = _host_roundtrip([Q, K, V])
         O_host, LSE_host, O, LSE = O, LSE, None, None
@@ -256,10 +273,12 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
         O = torch.empty_like(Q)
     if LSE is None and return_lse:
         LSE = torch.empty((B, Hq, Nq), dtype=torch.float32, device=Q.device)
-    dev = _one_device(Q, K, V, O, LSE, kept_terms)
+    if kcache_groups is not None:
+        _check_kcache_groups(kcache_groups, B, Hkv, N, d)
+    dev = _one_device(Q, K, V, O, LSE, kept_terms, kcache_groups)
     ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL, B, Hq, Hkv, N, d), Q.device)
     tab, _keep = _table_ptr(table, d)
-    o = _opts(mode, kept_terms, None)
+    o = _opts(mode, kept_terms, None, kcache_groups=kcache_groups)
     lse_ptr = C.c_void_p(LSE.data_ptr()) if LSE is not None else None
     with dev:
         if Nq == N:
@@ -277,7 +296,7 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
 
 
 def atf_prefill_host(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
-                     O=None, LSE=None, chunk_rows=0, device=None):
+                     O=None, LSE=None, chunk_rows=0, device=None, kcache_groups=None):
     """atf_prefill for HOST tensors (Q [B,Hq,N,d], K/V [B,Hkv,N,d] bf16, rotated): the C call copies,
     computes and copies back chunk by chunk on three streams.  Pinned tensors overlap; O / LSE, if
     given, are host tensors that receive the results (reuse pinned ones across calls).
@@ -302,7 +321,9 @@ def atf_prefill_host(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept
         raise AtfError(1, "unsupported shape")
     ws = ensure_workspace(need, device)  # the scratch starts with the workspace header the status check reads
     tab, _keep = _table_ptr(table, d)
-    o = _opts(mode, kept_terms, None)
+    if kcache_groups is not None:
+        _check_kcache_groups(kcache_groups, B, Hkv, N, d)
+    o = _opts(mode, kept_terms, None, kcache_groups=kcache_groups)
     with torch.cuda.device(device):
         stream = torch.cuda.current_stream(device)
         _check(lib().atf_prefill_host(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
@@ -344,19 +365,18 @@ def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=No
     Hkv, L = Vcache.shape[1], Vcache.shape[2]
     k_layout = ATF_KLAYOUT_GROUPS if Kcache.dim() == 6 else ATF_KLAYOUT_ROWS
     if k_layout == ATF_KLAYOUT_GROUPS:
-        kt = int(lib().atf_kcache_tile_keys(d))
-        want_k = (B, Hkv, (L + kt - 1) // kt, d // 16, kt, 16)
-    else:
-        want_k = (B, Hkv, L, d)
-    if Vcache.shape != (B, Hkv, L, d) or tuple(Kcache.shape) != want_k:
-        raise AtfError(1, "Vcache must be [B,Hkv,L,d] and Kcache [B,Hkv,L,d] or [B,Hkv,tiles,d/16,KT,16], matching q")
+        _check_kcache_groups(Kcache, B, Hkv, L, d)  # may be laid out for more keys than it holds yet
+    elif tuple(Kcache.shape) != (B, Hkv, L, d):
+        raise AtfError(1, "Kcache must be [B,Hkv,L,d] or a group-major cache [B,Hkv,tiles,d/16,KT,16], matching q")
+    if Vcache.shape != (B, Hkv, L, d):
+        raise AtfError(1, "Vcache must be [B,Hkv,L,d], matching q")
     if O is None:
         O = torch.empty_like(q)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
     dev = _one_device(q, Kcache, Vcache, O, kept_terms)
     ensure_workspace(atf_workspace_bytes(ATF_OP_DECODE, B, Hq, Hkv, L, d), q.device)
     tab, _keep = _table_ptr(table, d)
-    o = _opts(mode, kept_terms, lse, k_layout)
+    o = _opts(mode, kept_terms, lse, k_layout, kcache_groups=Kcache if k_layout == ATF_KLAYOUT_GROUPS else None)
     with dev:
         _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
                                    C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,

@@ -2,6 +2,7 @@
 // over the sm_100a instructions the kernels use (mbarrier, TMA, tcgen05 / tensor memory).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -42,11 +43,17 @@ AtfWorkspace atf_bound_workspace();
 // atf_check_status also reads (and clears) the status words registered here for the device
 void atf_register_status_words(int device, void* dev_ptr);
 
-// decode CTAs resident on the GPU at once: 2 per SM when K is read in the row layout, 3 per SM
-// with the group-major K cache (measured: whole-row streaming is fastest with fewer blocks in
-// flight, the sparser group-major reads want more)
+// Tiled TMA map of a [BH, N, D] bf16 tensor (heads head_rows rows apart): 64-column x box_rows boxes, 128-byte swizzle.
+atf_status atf_make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N, int D, int64_t head_rows,
+                             int box_rows);
+
+// decode CTAs resident on the GPU at once: 2 per SM in both layouts (the row-layout kernel keeps
+// four 2-stage cp.async rings per block, the tile kernel one 3-stage ring of 32 KiB stages)
 constexpr int ATF_DECODE_SLOTS_ROWS = 148 * 2;
-constexpr int ATF_DECODE_SLOTS_GROUPS = 148 * 3;
+#ifndef ATF_TL_CTAS
+#define ATF_TL_CTAS 2
+#endif
+constexpr int ATF_DECODE_SLOTS_GROUPS = 148 * ATF_TL_CTAS;
 constexpr int ATF_DECODE_MIN_SPLIT = 512;
 int atf_decode_num_splits(int B, int Hkv, int64_t L, int slots);
 
@@ -125,6 +132,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
+}
+// Untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion on an mbarrier.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");

@@ -53,9 +53,11 @@ struct DecodeParams {
   __nv_bfloat16* O;
   float* lse;                // may be null
   float* partials;           // [B*Hkv][nsplit][G][D + 2]
+  unsigned int* status;      // two status words of the workspace (give-up report)
   unsigned int* counters;    // [B*Hkv], zero between launches
   unsigned long long* kept;  // may be null
   int Hq, Hkv, G, L, nsplit;
+  int ktiles;                // group-major K cache: tiles per (batch, KV head), >= ceil(L / tile keys)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -86,8 +88,8 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-template <int D, int MODE, bool COUNT, int KL>
-__global__ void __launch_bounds__(DEC_THREADS, KL == ATF_KLAYOUT_ROWS ? 2 : 3)
+template <int D, int MODE, bool COUNT>
+__global__ void __launch_bounds__(DEC_THREADS, 2)
 atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant__ AtfTable table) {
   constexpr int H = D / 2;
   constexpr int CPR = D / 8;            // 16-byte chunks per cache row
@@ -98,7 +100,6 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   constexpr int NNT = D / 8;            // MMA N tiles of O
   constexpr int PSTRIDE = D + 2;        // floats per (split, head) partial: m, l, o[D]
   constexpr int CP_PER_LANE = KB * CPR / 32;
-  constexpr int KT = DEC_WARPS * KB;    // keys per tile of the group-major K cache (one block per warp)
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
 
   extern __shared__ __align__(128) uint8_t dsm[];
@@ -115,18 +116,13 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   const int m0 = split * (DEC_WARPS * KB);
   const int m1 = L;
   const int64_t slab = ((int64_t)b * P.Hkv + hkv) * (int64_t)L * D;
-  // the group-major cache is padded to whole tiles of DEC_WARPS * KB keys
-  const __nv_bfloat16* Kb = P.K + (KL == ATF_KLAYOUT_ROWS
-                                       ? slab
-                                       : ((int64_t)b * P.Hkv + hkv) * (((int64_t)L + DEC_WARPS * KB - 1) / (DEC_WARPS * KB)) *
-                                             (int64_t)(DEC_WARPS * KB) * D);
+  const __nv_bfloat16* Kb = P.K + slab;
   if (threadIdx.x < H) sW[threadIdx.x] = table.w[threadIdx.x];
   __syncthreads();
   const int Wmax = sW[H - 1];
 
-  // A fragments of q for every K step: rows = heads of the group (rows >= G stay zero).
-  // Row layout: K step j contracts dims 16j..16j+15.  Group-major layout: K step j contracts the
-  // 8 pairs of group j, lowest frequency first, each pair as (dim r, dim r + h) side by side.
+  // A fragments of q for every K step: rows = heads of the group (rows >= G stay zero); K step j
+  // contracts dims 16j..16j+15.
   uint32_t qa[NKS][2];
 #pragma unroll
   for (int j = 0; j < NKS; ++j) {
@@ -134,37 +130,24 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
     qa[j][1] = 0u;
     if (g < G) {
       const __nv_bfloat16* qrow = P.q + ((int64_t)b * P.Hq + hkv * G + g) * D;
-      if (KL == ATF_KLAYOUT_ROWS) {
-        qa[j][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t);
-        qa[j][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 8 + 2 * t);
-      } else {
-        const int ra = H - 1 - (8 * j + t), rb = H - 1 - (8 * j + 4 + t);
-        const uint16_t* q16 = reinterpret_cast<const uint16_t*>(qrow);
-        qa[j][0] = (uint32_t)q16[ra] | ((uint32_t)q16[ra + H] << 16);
-        qa[j][1] = (uint32_t)q16[rb] | ((uint32_t)q16[rb + H] << 16);
-      }
+      qa[j][0] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t);
+      qa[j][1] = *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 8 + 2 * t);
     }
   }
 
   // ---- copy and fragment addressing, fixed per lane ----
   constexpr int PITCH = ROWB + 16;          // shared-memory row pitch of a row-layout block
   constexpr int RSTEP = 32 / CPR;           // rows covered by one warp-wide copy
-  constexpr int GSZ = KB * 36;              // shared-memory bytes of one group of a group-major K block
-  static_assert(KB * PITCH <= DEC_TILE_SMEM && NKS * GSZ <= DEC_TILE_SMEM, "block does not fit its shared-memory tile");
+  static_assert(KB * PITCH <= DEC_TILE_SMEM, "block does not fit its shared-memory tile");
   const int cp_chunk = lane % CPR;          // this lane's 16-byte chunk of a cache row
   const int cp_row0 = lane / CPR;           // first row this lane copies; then every RSTEP rows
   const uint32_t cp_dst0 = cp_row0 * PITCH + cp_chunk * 16;
-  const int gk_row = lane >> 1, gk_half = lane & 1;  // group-major K: (key, half of its 32 bytes) of a 16-key copy
-  const uint32_t gk_dst0 = gk_row * 32 + (gk_row >> 2) * 16 + gk_half * 16;
   const uint32_t warp_smem = smem_u32(dsm) + warp * DEC_WARP_SMEM;
   const int lm_i = lane >> 3, lm_r = lane & 7;  // ldmatrix: matrix fed by this lane and row in it
-  const uint32_t k_lane_off = KL == ATF_KLAYOUT_ROWS
-                                  ? ((lm_i >> 1) * 8 + lm_r) * PITCH + (lm_i & 1) * 16
-                                  : ((lm_i >> 1) * 8 + lm_r) * 32 + ((((lm_i >> 1) * 8 + lm_r) >> 2) * 16) + (lm_i & 1) * 16;
+  const uint32_t k_lane_off = ((lm_i >> 1) * 8 + lm_r) * PITCH + (lm_i & 1) * 16;
   const uint32_t v_lane_off = ((lm_i & 1) * 8 + lm_r) * PITCH + (lm_i >> 1) * 16;
 
   const __nv_bfloat16* Vb = P.V + slab;
-  int r_iss = 0;  // cursor for the copies: first live pair of the nearest key of the block being fetched
   auto issue_block = [&](int kb0, int stage) {
     const uint32_t ks = warp_smem + stage * DEC_STAGE_SMEM, vs = ks + DEC_TILE_SMEM;
     // every key of the block exists and is reached by some pair: no predicates
@@ -176,7 +159,7 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
       const int64_t goff = (int64_t)(kb0 + cp_row0) * D + cp_chunk * 8;
 #pragma unroll
       for (int i = 0; i < CP_PER_LANE; ++i) {
-        if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff + i * RSTEP * D, 16);
+        cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff + i * RSTEP * D, 16);
         cp_async16(vs + cp_dst0 + i * RSTEP * PITCH, Vb + goff + i * RSTEP * D, 16);
       }
     } else {
@@ -186,33 +169,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
         const bool valid = key < m1 && (L - 1 - key) <= Wmax;
         const int keyc = key < m1 ? key : m1 - 1;
         const int64_t goff = (int64_t)keyc * D + cp_chunk * 8;
-        if (KL == ATF_KLAYOUT_ROWS) cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff, valid ? 16 : 0);
+        cp_async16(ks + cp_dst0 + i * RSTEP * PITCH, Kb + goff, valid ? 16 : 0);
         cp_async16(vs + cp_dst0 + i * RSTEP * PITCH, Vb + goff, valid ? 16 : 0);
-      }
-    }
-    if (KL == ATF_KLAYOUT_GROUPS) {
-      // group-major K: the live pairs of a key are its first groups, each group a contiguous
-      // stream over the keys of the tile, so only live bytes are fetched (8-pair granularity)
-      const int z_near = max(L - 1 - (kb0 + KB - 1), 0);
-      if (r_iss >= H || sW[r_iss] < z_near) {
-        r_iss = 0;
-        while (r_iss < H && sW[r_iss] < z_near) ++r_iss;
-      } else {
-        while (r_iss > 0 && sW[r_iss - 1] >= z_near) --r_iss;
-      }
-      const int ngl = (H - r_iss + 7) >> 3;  // live groups of the nearest key
-      const int64_t tile0 = ((int64_t)(kb0 / KT) * NKS * KT + (kb0 % KT)) * 16;  // group 0, first key of the block
-#pragma unroll
-      for (int gi = 0; gi < NKS; ++gi) {
-        if (gi < ngl) {
-#pragma unroll
-          for (int i = 0; i < KB / 16; ++i) {
-            const int key = kb0 + i * 16 + gk_row;
-            const bool valid = key < m1;
-            const int64_t goff = tile0 + ((int64_t)gi * KT + (valid ? i * 16 + gk_row : 0)) * 16 + gk_half * 8;
-            cp_async16(ks + gi * GSZ + i * 576 + gk_dst0, Kb + goff, valid ? 16 : 0);
-          }
-        }
       }
     }
   };
@@ -280,8 +238,8 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
 #pragma unroll
       for (int e = 0; e < 4; ++e) sc[kg][e] = 0.f;
 
-    if (KL == ATF_KLAYOUT_ROWS) {
-      // ---- S = q K^T, row layout ----
+    {
+      // ---- S = q K^T ----
       // K steps (16 pairs of one half) below the nearest key's first live pair are dead for every key
       const int jl = rq_near >> 4;
       // element masks of the K step that holds a first live pair r: lane t holds pairs 2t, 2t+1 of the
@@ -323,28 +281,6 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
               bf[2 * h2] &= mk0;
               bf[2 * h2 + 1] &= mk1;
             }
-          }
-          mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
-          mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
-        }
-      }
-    } else {
-      // ---- S = q K^T, group-major layout: K step j = the 8 pairs of group j; a key with first
-      //      live pair r keeps its first H - r pairs in this order ----
-      const int ngl = (H - rq_near + 7) >> 3;  // groups fetched for this block
-#pragma unroll
-      for (int j = 0; j < NKS; ++j) {
-        if (j >= ngl) continue;  // warp-uniform
-#pragma unroll
-        for (int kp = 0; kp < NKG / 2; ++kp) {
-          // matrices: (keys of group 2kp, first half), (same, second half), (keys of group 2kp+1, ...)
-          uint32_t bf[4];
-          ldsm_x4(ks + k_lane_off + j * GSZ + kp * 576, bf);
-#pragma unroll
-          for (int h2 = 0; h2 < 2; ++h2) {
-            const int live = H - r_lane[2 * kp + h2];  // pairs this lane's key keeps
-            if (8 * j + t >= live) bf[2 * h2] = 0u;
-            if (8 * j + 4 + t >= live) bf[2 * h2 + 1] = 0u;
           }
           mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
           mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
@@ -517,9 +453,370 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
   if (threadIdx.x == 0) P.counters[grp] = 0;  // ready for the next launch
 }
 
+// ------------------------------------------------------------------------------------------
+// Decode on the tiled group-major K cache: bulk copies instead of per-lane 16-byte copies.
+//
+// A tile is KT keys (16 KiB of K, 16 KiB of V).  In the cache a K tile is [group of 8 pairs, lowest
+// frequency first][key][16 elements], so the pairs the tile's nearest key keeps are a contiguous
+// prefix of the tile: ONE untiled bulk copy fetches exactly the live bytes.  The two 16-byte
+// halves of a key's group entry are stored swapped for keys with bit 2 set, which makes the
+// ldmatrix reads of the copied image free of bank conflicts without padding.  The V tile (rows of
+// the ordinary cache) comes by TMA with the 128-byte swizzle for the same reason.
+// Block = 4 consumer warps (a quarter of the tile each, the arithmetic of the row-layout kernel)
+// + 1 producer warp (one thread issues the copies of the next tiles into a 3-stage ring; full and
+// empty mbarriers per stage, every wait bounded).
+// ------------------------------------------------------------------------------------------
+#ifndef ATF_TL_STAGES
+#define ATF_TL_STAGES 3
+#endif
+constexpr int TL_STAGES = ATF_TL_STAGES;
+constexpr int TL_THREADS = (DEC_WARPS + 1) * 32;
+constexpr int TL_TILE_BYTES = 16384;
+constexpr int TL_STAGE_BYTES = 2 * TL_TILE_BYTES;
+constexpr int TL_SMEM = TL_STAGES * TL_STAGE_BYTES + 1024 /* alignment slack */ + 64 /* barriers */;
+
+template <int D, int MODE, bool COUNT>
+__global__ void __launch_bounds__(TL_THREADS, ATF_DECODE_SLOTS_GROUPS / 148)
+atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ DecodeParams P,
+                        const __grid_constant__ AtfTable table) {
+  constexpr int H = D / 2;
+  constexpr int KT = TL_TILE_BYTES / (D * 2);  // keys per tile (64 for d = 128, 128 for d = 64)
+  constexpr int KB = KT / DEC_WARPS;            // keys per consumer warp and tile
+  constexpr int NKG = KB / 8;
+  constexpr int NKS = D / 16;                   // groups of 8 pairs = MMA K steps of q K^T
+  constexpr int NNT = D / 8;
+  constexpr int NVB = D / 64;                   // 64-column boxes of a V tile
+  constexpr int PSTRIDE = D + 2;
+  constexpr int GBYTES = KT * 32;               // one group of a K tile
+  const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
+
+  extern __shared__ uint8_t dsm_raw[];
+  __shared__ int sW[ATF_MAX_PAIRS];
+  __shared__ unsigned int s_last;
+  __shared__ int s_abort;
+  const uint32_t sbase = (smem_u32(dsm_raw) + 1023u) & ~1023u;
+  uint8_t* sgen = dsm_raw + (sbase - smem_u32(dsm_raw));
+  const uint32_t bars = sbase + TL_STAGES * TL_STAGE_BYTES;
+  auto full_bar = [&](int st) { return bars + 8u * (uint32_t)st; };
+  auto empty_bar = [&](int st) { return bars + 8u * (uint32_t)(TL_STAGES + st); };
+
+  const int split = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t4 = lane & 3;
+  const int G = P.G, L = P.L;
+  const int64_t grp = (int64_t)b * P.Hkv + hkv;
+  const int ntiles = (L + KT - 1) / KT;
+  if (threadIdx.x < H) sW[threadIdx.x] = table.w[threadIdx.x];
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int st = 0; st < TL_STAGES; ++st) {
+      mbar_init(full_bar(st), 1);
+      mbar_init(empty_bar(st), DEC_WARPS);
+    }
+    mbar_fence_init();
+    fence_proxy_async_smem();
+    tma_prefetch_desc(&tmV);
+  }
+  __syncthreads();
+  const int Wmax = sW[H - 1];
+  // the first tile that holds a key some pair reaches; tiles are dealt round-robin to the splits
+  const int t_lo = max(0, L - 1 - Wmax) / KT;
+  const int t_first = t_lo + split;
+  const __nv_bfloat16* Kb = P.K + grp * (int64_t)P.ktiles * KT * D;
+  unsigned int fail_site = 0;
+  volatile int* abortp = &s_abort;
+  auto bounded_wait = [&](uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+      for (int i = 0; i < 128; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+      if (*abortp) return false;
+      if (global_timer_ns() - t0 > ATF_WAIT_LIMIT_NS) {
+        *abortp = 1;
+        return false;
+      }
+    }
+  };
+
+  float oacc[NNT][4];
+#pragma unroll
+  for (int nt = 0; nt < NNT; ++nt)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[nt][e] = 0.f;
+  float m_used = -INFINITY, l_part = 0.f;
+  unsigned long long cnt = 0;
+
+  if (warp == DEC_WARPS) {
+    // =============================== producer ===============================
+    if (lane == 0) {
+      int r_near = 0;  // first live pair of the tile's nearest key: only moves down as the tiles advance
+      {
+        const int z0 = max(L - 1 - (t_first * KT + KT - 1), 0);
+        while (r_near < H && sW[r_near] < z0) ++r_near;
+      }
+      int it = 0;
+      for (int t = t_first; t < ntiles; t += P.nsplit, ++it) {
+        const int st = it % TL_STAGES;
+        if (it >= TL_STAGES && !bounded_wait(empty_bar(st), ((it / TL_STAGES) - 1) & 1)) { fail_site = 40; break; }
+        const int z_near = max(L - 1 - (t * KT + KT - 1), 0);
+        while (r_near > 0 && sW[r_near - 1] >= z_near) --r_near;
+        const int rq = MODE == ATF_MODE_COARSE ? (r_near & ~7) : r_near;
+        const int ngl = (H - rq + 7) >> 3;  // live groups of the nearest key: the prefix to fetch
+        const uint32_t kdst = sbase + st * TL_STAGE_BYTES, vdst = kdst + TL_TILE_BYTES;
+        mbar_expect_tx(full_bar(st), (uint32_t)(ngl * GBYTES + TL_TILE_BYTES));
+        bulk_load_1d(kdst, Kb + (int64_t)t * KT * D, (uint32_t)(ngl * GBYTES), full_bar(st));
+#pragma unroll
+        for (int vb = 0; vb < NVB; ++vb)
+          tma_load_3d(vdst + vb * (KT * 128), &tmV, full_bar(st), vb * 64, t * KT, (int)grp);
+      }
+    }
+  } else {
+    // =============================== consumers ===============================
+    // A fragments of q: K step j contracts the 8 pairs of group j, each pair as (dim r, dim r + h)
+    uint32_t qa[NKS][2];
+#pragma unroll
+    for (int j = 0; j < NKS; ++j) {
+      qa[j][0] = 0u;
+      qa[j][1] = 0u;
+      if (g < G) {
+        const uint16_t* q16 = reinterpret_cast<const uint16_t*>(P.q + ((int64_t)b * P.Hq + hkv * G + g) * D);
+        const int ra = H - 1 - (8 * j + t4), rb = H - 1 - (8 * j + 4 + t4);
+        qa[j][0] = (uint32_t)q16[ra] | ((uint32_t)q16[ra + H] << 16);
+        qa[j][1] = (uint32_t)q16[rb] | ((uint32_t)q16[rb + H] << 16);
+      }
+    }
+    const int lm_i = lane >> 3, lm_r = lane & 7;
+    // K: matrices (keys 0-7 first half), (keys 0-7 second half), (keys 8-15 first half), (keys 8-15 second half)
+    const int kkey = warp * KB + (lm_i >> 1) * 8 + lm_r;  // + 16 * kp
+    const uint32_t k_lane_off = (uint32_t)kkey * 32u + (uint32_t)(((lm_i & 1) ^ ((kkey >> 2) & 1)) << 4);
+    // V: matrices (keys 0-7, chunk 2np), (keys 8-15, chunk 2np), (keys 0-7, chunk 2np+1), (keys 8-15, chunk 2np+1)
+    const int vrow = warp * KB + (lm_i & 1) * 8 + lm_r;  // + 16 * pk
+    const uint32_t v_row_off = (uint32_t)vrow * 128u;
+    int r_far = 0;
+    {
+      const int z0 = L - 1 - (t_first * KT + warp * KB);
+      while (r_far < H && sW[r_far] < z0) ++r_far;
+    }
+    int it = 0;
+    for (int t = t_first; t < ntiles; t += P.nsplit, ++it) {
+      const int st = it % TL_STAGES;
+      if (!bounded_wait(full_bar(st), (it / TL_STAGES) & 1)) { fail_site = 41; break; }
+      const uint32_t ks = sbase + st * TL_STAGE_BYTES, vs = ks + TL_TILE_BYTES;
+      const int kb0 = t * KT + warp * KB;
+      const bool blk_fast = (kb0 + KB <= L) && (L - 1 - kb0 <= Wmax);
+
+      // ---- live pair range over the warp's keys (coarse mode: first live pair rounded down to 8) ----
+      const int z_far = L - 1 - kb0;
+      const int z_near = max(L - 1 - (kb0 + KB - 1), 0);
+      while (r_far > 0 && sW[r_far - 1] >= z_far) --r_far;
+      int r_near = r_far;
+      while (r_near > 0 && sW[r_near - 1] >= z_near) --r_near;
+      const int rq_far = MODE == ATF_MODE_COARSE ? (r_far >= H ? H : (r_far & ~7)) : r_far;
+      const int rq_near = MODE == ATF_MODE_COARSE ? (r_near & ~7) : r_near;
+      int r_lane[NKG];
+#pragma unroll
+      for (int kg = 0; kg < NKG; ++kg) r_lane[kg] = rq_far;
+      if (rq_near != rq_far) {
+#pragma unroll
+        for (int kg = 0; kg < NKG; ++kg) {
+          const int z = L - 1 - (kb0 + kg * 8 + g);
+          int r = r_near;
+          while (r < r_far && sW[r] < z) ++r;
+          r_lane[kg] = MODE == ATF_MODE_COARSE ? (r >= H ? H : (r & ~7)) : r;
+        }
+      }
+      float sc[NKG][4];
+#pragma unroll
+      for (int kg = 0; kg < NKG; ++kg)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sc[kg][e] = 0.f;
+
+      // ---- S = q K^T: K step j = the 8 pairs of group j; a key with first live pair r keeps its first H - r pairs ----
+      const int ngl = (H - rq_near + 7) >> 3;
+#pragma unroll
+      for (int j = 0; j < NKS; ++j) {
+        if (j >= ngl) continue;  // warp-uniform
+#pragma unroll
+        for (int kp = 0; kp < NKG / 2; ++kp) {
+          uint32_t bf[4];
+          ldsm_x4(ks + j * GBYTES + kp * 512 + k_lane_off, bf);
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int live = H - r_lane[2 * kp + h2];
+            if (8 * j + t4 >= live) bf[2 * h2] = 0u;
+            if (8 * j + 4 + t4 >= live) bf[2 * h2 + 1] = 0u;
+          }
+          mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
+          mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
+        }
+      }
+      if (COUNT && t4 == 0) {
+#pragma unroll
+        for (int kg = 0; kg < NKG; ++kg)
+          if (kb0 + kg * 8 + g < L) cnt += (unsigned long long)(H - r_lane[kg]);
+      }
+
+      // ---- online softmax (log2 domain); this lane holds keys 2t, 2t+1 of every group of 8 keys for head g ----
+      float mx = -INFINITY;
+      if (blk_fast) {
+#pragma unroll
+        for (int kg = 0; kg < NKG; ++kg)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            sc[kg][e] *= kScaleLog2;
+            mx = fmaxf(mx, sc[kg][e]);
+          }
+      } else {
+#pragma unroll
+        for (int kg = 0; kg < NKG; ++kg)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int key = kb0 + kg * 8 + 2 * t4 + e;
+            sc[kg][e] = (key < L && L - 1 - key <= Wmax) ? sc[kg][e] * kScaleLog2 : -INFINITY;
+            mx = fmaxf(mx, sc[kg][e]);
+          }
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      float scale_o = 1.f;
+      bool moved = false;
+      if (mx > m_used + (m_used == -INFINITY ? 0.f : DEC_RESCALE_THRESHOLD)) {
+        scale_o = (m_used == -INFINITY) ? 0.f : ex2f(m_used - mx);
+        m_used = mx;
+        moved = true;
+      }
+      if (__any_sync(0xffffffffu, moved)) {
+        l_part *= scale_o;
+#pragma unroll
+        for (int nt = 0; nt < NNT; ++nt) {
+          oacc[nt][0] *= scale_o;
+          oacc[nt][1] *= scale_o;
+        }
+      }
+      const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+      uint32_t pa[NKG];
+#pragma unroll
+      for (int kg = 0; kg < NKG; ++kg) {
+        const float p0 = ex2f(sc[kg][0] - mref), p1 = ex2f(sc[kg][1] - mref);
+        l_part += p0 + p1;
+        pa[kg] = pack_bf16x2(p0, p1);
+      }
+
+      // ---- O += P V (V tile in 128-byte-swizzled 64-column boxes) ----
+#pragma unroll
+      for (int pk = 0; pk < NKG / 2; ++pk) {
+#pragma unroll
+        for (int np = 0; np < NNT / 2; ++np) {
+          const int chunk = 2 * np + (lm_i >> 1);  // 16-byte column chunk of the row, 0 .. D/8 - 1
+          uint32_t bf[4];
+          ldsm_x4_trans(vs + (chunk >> 3) * (KT * 128) + pk * 2048 + v_row_off + (((chunk & 7) ^ lm_r) << 4), bf);
+          mma_bf16_16816(oacc[2 * np], pa[2 * pk], pa[2 * pk + 1], bf[0], bf[1]);
+          mma_bf16_16816(oacc[2 * np + 1], pa[2 * pk], pa[2 * pk + 1], bf[2], bf[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar(st));
+    }
+  }
+
+  // ---- merge the warps of the block (the ring is free once everybody is here) ----
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+  l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+  if (fail_site) {
+    atomicExch(P.status, 1u);
+    atomicExch(P.status + 1, fail_site);
+  }
+  __syncthreads();
+  float* sm = reinterpret_cast<float*>(sgen);  // [DEC_WARPS][G][PSTRIDE]
+  if (warp < DEC_WARPS && g < G) {
+    float* dst = sm + (warp * G + g) * PSTRIDE;
+    if (t4 == 0) {
+      dst[0] = m_used;
+      dst[1] = l_part;
+    }
+#pragma unroll
+    for (int nt = 0; nt < NNT; ++nt) {
+      dst[2 + nt * 8 + 2 * t4] = oacc[nt][0];
+      dst[2 + nt * 8 + 2 * t4 + 1] = oacc[nt][1];
+    }
+  }
+  __syncthreads();
+  float* part = P.partials + (grp * P.nsplit + split) * (int64_t)(G * PSTRIDE);
+  for (int idx = threadIdx.x; idx < G * D; idx += TL_THREADS) {
+    const int gg = idx / D, col = idx % D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm[(w * G + gg) * PSTRIDE]);
+    const float Ms = (M == -INFINITY) ? 0.f : M;
+    float acc = 0.f, lacc = 0.f;
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) {
+      const float* src = sm + (w * G + gg) * PSTRIDE;
+      const float f = ex2f(src[0] - Ms);
+      acc += f * src[2 + col];
+      lacc += f * src[1];
+    }
+    part[gg * PSTRIDE + 2 + col] = acc;
+    if (col == 0) {
+      part[gg * PSTRIDE] = M;
+      part[gg * PSTRIDE + 1] = lacc;
+    }
+  }
+  if (COUNT && warp < DEC_WARPS) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+    if (lane == 0 && cnt) {
+      for (int gg = 0; gg < G; ++gg) atomicAdd(P.kept + (int64_t)b * P.Hq + hkv * G + gg, cnt);
+    }
+  }
+
+  // ---- last block of this (batch, KV head) merges all splits ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int done = atomicAdd(P.counters + grp, 1u);
+    s_last = (done == (unsigned)P.nsplit - 1) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float* allp = P.partials + grp * P.nsplit * (int64_t)(G * PSTRIDE);
+  for (int gg = warp; gg < G; gg += DEC_WARPS + 1) {
+    float M = -INFINITY;
+    for (int sp = lane; sp < P.nsplit; sp += 32) M = fmaxf(M, __ldcg(allp + ((int64_t)sp * G + gg) * PSTRIDE));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    const float Ms = (M == -INFINITY) ? 0.f : M;
+    float Lsum = 0.f;
+    for (int sp = lane; sp < P.nsplit; sp += 32) {
+      const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
+      Lsum += ex2f(__ldcg(src) - Ms) * __ldcg(src + 1);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, off);
+    const float inv = 1.f / Lsum;
+    float acc[D / 32];
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+    for (int sp = 0; sp < P.nsplit; ++sp) {
+      const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
+      const float f = ex2f(__ldcg(src) - Ms);
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) acc[c] = fmaf(f, __ldcg(src + 2 + c * 32 + lane), acc[c]);
+    }
+    const int64_t hq = (int64_t)b * P.Hq + hkv * G + gg;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) P.O[hq * D + c * 32 + lane] = __float2bfloat16_rn(acc[c] * inv);
+    if (P.lse && lane == 0) P.lse[hq] = (Ms + log2f(Lsum)) * 0.6931471805599453f;
+  }
+  if (threadIdx.x == 0) P.counters[grp] = 0;  // ready for the next launch
+}
+
 // K cache rows -> tiled group-major order [slab][tile][group][key in tile][16].  One thread per
 // (key, group of 8 pairs): gathers the 16 elements of the group (pair p = 8*group + i is dims
-// h-1-p and d-1-p) and writes 32 bytes.
+// h-1-p and d-1-p) and writes 32 bytes (the two 16-byte halves swapped for keys with bit 2 set).
 __global__ void __launch_bounds__(256)
 atf_kcache_pack_kernel(const __nv_bfloat16* __restrict__ K, __nv_bfloat16* __restrict__ Kg, int64_t slabs, int64_t n,
                        int64_t ntiles, int64_t pos0, int D) {
@@ -539,17 +836,18 @@ atf_kcache_pack_kernel(const __nv_bfloat16* __restrict__ K, __nv_bfloat16* __res
   }
   const int64_t pos = pos0 + m, tile = pos / KT, kin = pos % KT;
   uint4* dst = reinterpret_cast<uint4*>(Kg + (((sl * ntiles + tile) * NG + gi) * KT + kin) * 16);
-  dst[0] = reinterpret_cast<const uint4*>(out)[0];
-  dst[1] = reinterpret_cast<const uint4*>(out)[1];
+  const int swap = (int)((kin >> 2) & 1);  // keys with bit 2 set store their two 16-byte halves swapped
+  dst[swap] = reinterpret_cast<const uint4*>(out)[0];
+  dst[swap ^ 1] = reinterpret_cast<const uint4*>(out)[1];
 }
 
-template <int D, int KL>
+template <int D>
 atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
   dim3 grid(P.nsplit, P.Hkv, B);
 #define ATF_DEC_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                  \
-    auto kern = atf_decode_kernel<D, MODE_, COUNT_, KL>;                                                    \
-    const int smem = KL == ATF_KLAYOUT_ROWS ? DEC_SMEM_ROWS : DEC_SMEM;                                 \
+    auto kern = atf_decode_kernel<D, MODE_, COUNT_>;                                                    \
+    const int smem = DEC_SMEM_ROWS;                                                                     \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));      \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,           \
                                         cudaSharedmemCarveoutMaxShared));                                \
@@ -561,6 +859,28 @@ atf_status launch_decode(const DecodeParams& P, const AtfTable& t, int B, int mo
     if (count) ATF_DEC_LAUNCH(ATF_MODE_COARSE, true); else ATF_DEC_LAUNCH(ATF_MODE_COARSE, false);
   }
 #undef ATF_DEC_LAUNCH
+  ATF_CUDA_CHECK(cudaGetLastError());
+  return ATF_OK;
+}
+
+template <int D>
+atf_status launch_decode_tiles(const CUtensorMap& tmV, const DecodeParams& P, const AtfTable& t, int B, int mode, bool count,
+                               cudaStream_t s) {
+  dim3 grid(P.nsplit, P.Hkv, B);
+#define ATF_TL_LAUNCH(MODE_, COUNT_)                                                                        \
+  do {                                                                                                      \
+    auto kern = atf_decode_tiles_kernel<D, MODE_, COUNT_>;                                                  \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TL_SMEM));       \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,               \
+                                        cudaSharedmemCarveoutMaxShared));                                    \
+    kern<<<grid, TL_THREADS, TL_SMEM, s>>>(tmV, P, t);                                                      \
+  } while (0)
+  if (mode == ATF_MODE_EXACT) {
+    if (count) ATF_TL_LAUNCH(ATF_MODE_EXACT, true); else ATF_TL_LAUNCH(ATF_MODE_EXACT, false);
+  } else {
+    if (count) ATF_TL_LAUNCH(ATF_MODE_COARSE, true); else ATF_TL_LAUNCH(ATF_MODE_COARSE, false);
+  }
+#undef ATF_TL_LAUNCH
   ATF_CUDA_CHECK(cudaGetLastError());
   return ATF_OK;
 }
@@ -620,7 +940,12 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   const int64_t kt = DEC_WARPS * (DEC_TILE_BYTES / (d * 2));  // keys per tile; tiles go round-robin to the splits
   const int64_t ntiles = (L + kt - 1) / kt;
   if (P.nsplit > ntiles) P.nsplit = (int)ntiles;
+  // a group-major cache laid out for more keys than it holds yet (room for the tokens to come)
+  const int64_t cap = (opts && opts->kcache_capacity > 0) ? opts->kcache_capacity : L;
+  if (cap < L) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: kcache_capacity (%lld) is smaller than L", (long long)cap);
+  P.ktiles = (int)((cap + kt - 1) / kt);
   char* base = (char*)ws.ptr;
+  P.status = (unsigned int*)base;
   P.counters = (unsigned int*)(base + ATF_WS_STATUS_BYTES);
   P.partials = (float*)(base + ATF_WS_HEADER);
   cudaStream_t s = (cudaStream_t)stream;
@@ -628,10 +953,11 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   const int kl = opts ? opts->k_layout : ATF_KLAYOUT_ROWS;
   if (kl != ATF_KLAYOUT_ROWS && kl != ATF_KLAYOUT_GROUPS) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: unknown k_layout %d", kl);
   if (kl == ATF_KLAYOUT_ROWS)
-    return d == 64 ? launch_decode<64, ATF_KLAYOUT_ROWS>(P, t, B, mode, count, s)
-                   : launch_decode<128, ATF_KLAYOUT_ROWS>(P, t, B, mode, count, s);
-  return d == 64 ? launch_decode<64, ATF_KLAYOUT_GROUPS>(P, t, B, mode, count, s)
-                 : launch_decode<128, ATF_KLAYOUT_GROUPS>(P, t, B, mode, count, s);
+    return d == 64 ? launch_decode<64>(P, t, B, mode, count, s) : launch_decode<128>(P, t, B, mode, count, s);
+  // tiled group-major K cache: bulk copies of the live prefix of each K tile, V tiles by TMA
+  CUtensorMap tmV;
+  if ((st = atf_make_tile_map(&tmV, Vcache, (int64_t)B * Hkv, L, d, L, (int)kt)) != ATF_OK) return st;
+  return d == 64 ? launch_decode_tiles<64>(tmV, P, t, B, mode, count, s) : launch_decode_tiles<128>(tmV, P, t, B, mode, count, s);
 }
 
 extern "C" int64_t atf_kcache_tile_keys(int d) { return (d == 64 || d == 128) ? DEC_WARPS * (DEC_TILE_BYTES / (d * 2)) : 0; }

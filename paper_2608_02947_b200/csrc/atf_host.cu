@@ -1,5 +1,7 @@
 // Host-side parts of the atflash library: window table (Eq. 2, Eq. 3, Sec. 3.2), error
 // text, workspace binding and the device status word.
+#include <cuda.h>
+
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -26,6 +28,39 @@ atf_status atf_fail(atf_status code, const char* fmt, ...) {
 }
 
 AtfWorkspace atf_bound_workspace() { return g_ws; }
+
+// ---- tiled tensor maps for TMA ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+  if (qres != cudaDriverEntryPointSuccess) return nullptr;
+  fn = (EncodeTiledFn)p;
+  return fn;
+}
+
+// [BH, N, D] bf16 tensor whose heads are head_rows (>= N) rows apart in memory; box = 64 columns x
+// box_rows rows x 1, 128-byte swizzle, zero fill outside.
+atf_status atf_make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N, int D, int64_t head_rows,
+                             int box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return atf_fail(ATF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)head_rows * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return atf_fail(ATF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return ATF_OK;
+}
 
 // Splits of the key range per (batch, KV head) for decode: the smallest split count that fills
 // whole waves of the `slots` resident CTAs best, with at least ATF_DECODE_MIN_SPLIT keys per split.

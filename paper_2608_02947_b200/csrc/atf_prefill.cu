@@ -97,9 +97,12 @@ constexpr int HK = T / 2;  // keys per half tile: S and P are produced and consu
 
 __global__ void __launch_bounds__(256)
 atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict__ Y, int64_t rows, int D,
-                  int64_t n_per_head, int64_t src_head_rows) {
+                  int64_t n_per_head, int64_t src_head_rows, __nv_bfloat16* __restrict__ Kg, int64_t kg_tiles,
+                  int64_t kg_first_row) {
   // one thread writes 8 consecutive output columns (4 pairs) of one row; the source holds
-  // src_head_rows rows per head of which the first n_per_head are copied, the result is dense
+  // src_head_rows rows per head of which the first n_per_head are copied, the result is dense.
+  // With Kg the same 16 bytes also go into the tiled group-major K cache (kg_tiles tiles per head), for
+  // the rows from kg_first_row on: a group of that cache is two such 16-byte pieces of a key.
   const int H = D / 2;
   const int per_row = D / 8;
   const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -107,7 +110,8 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
   const int64_t row = gid / per_row;
   const int t = (int)(gid % per_row);
   const int64_t head = row / n_per_head;
-  const __nv_bfloat16* src = X + (head * src_head_rows + (row - head * n_per_head)) * D;
+  const int64_t m = row - head * n_per_head;  // position of the row in its head
+  const __nv_bfloat16* src = X + (head * src_head_rows + m) * D;
   __align__(16) __nv_bfloat16 out[8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -116,6 +120,13 @@ atf_repack_kernel(const __nv_bfloat16* __restrict__ X, __nv_bfloat16* __restrict
     out[2 * i + 1] = src[D - 1 - p];
   }
   *reinterpret_cast<uint4*>(Y + row * D + 8 * t) = *reinterpret_cast<const uint4*>(out);
+  if (Kg && m >= kg_first_row) {
+    const int64_t KT = 8192 / D;  // keys per 16 KiB tile
+    const int64_t tile = m / KT, kin = m % KT;
+    const int j = t >> 1, half = (t & 1) ^ (int)((kin >> 2) & 1);
+    *reinterpret_cast<uint4*>(Kg + (((head * kg_tiles + tile) * (D / 16) + j) * KT + kin) * 16 + half * 8) =
+        *reinterpret_cast<const uint4*>(out);
+  }
 }
 
 // Band schedule word of (tile distance dt, row quarter wq), tiles of 128 aligned at 0.  The 32
@@ -830,37 +841,6 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 }
 
 // ---- host ----
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn) return fn;
-  void* p = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
-  if (qres != cudaDriverEntryPointSuccess) return nullptr;
-  fn = (EncodeTiledFn)p;
-  return fn;
-}
-
-// [BH, N, D] bf16 tensor, box = 64 columns x 128 rows x 1, 128-byte swizzle, zero fill outside.
-atf_status make_tile_map(CUtensorMap* m, const void* base, int64_t BH, int64_t N, int D, int64_t head_rows = 0) {
-  if (head_rows == 0) head_rows = N;  // rows between two heads in memory (>= N)
-  EncodeTiledFn enc = get_encode_fn();
-  if (!enc) return atf_fail(ATF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)head_rows * D * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)T, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return atf_fail(ATF_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-  return ATF_OK;
-}
-
 template <int D>
 atf_status launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& P,
                           const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
@@ -922,6 +902,10 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
     return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: pointers must be 16-byte aligned");
   const int mode = opts ? opts->mode : ATF_MODE_EXACT;
   if (mode != ATF_MODE_EXACT && mode != ATF_MODE_COARSE) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: unknown mode %d", mode);
+  if (opts && opts->kcache_groups) {
+    if (opts->kcache_capacity < N) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: kcache_capacity (%lld) is smaller than N", (long long)opts->kcache_capacity);
+    if ((uintptr_t)opts->kcache_groups & 15) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill: kcache_groups must be 16-byte aligned");
+  }
   AtfTable t;
   atf_status st = atf_validate_table("atf_prefill", table, d, N, &t);
   if (st != ATF_OK) return st;
@@ -951,15 +935,19 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
     const int64_t rows_q = (int64_t)B * Hq * Nq, rows_k = (int64_t)B * Hkv * N;
     const int64_t bq = (rows_q * (d / 8) + 255) / 256, bk = (rows_k * (d / 8) + 255) / 256;
     if (bq > 0x7FFFFFFF) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill: problem too large for the repack grid");
-    atf_repack_kernel<<<(unsigned)bq, 256, 0, s>>>((const __nv_bfloat16*)Q, Qp, rows_q, d, Nq, Nq);
-    atf_repack_kernel<<<(unsigned)bk, 256, 0, s>>>((const __nv_bfloat16*)K, Kp, rows_k, d, N, kv_head_rows);
+    __nv_bfloat16* Kg = opts ? (__nv_bfloat16*)opts->kcache_groups : nullptr;
+    const int64_t kt = 8192 / d;
+    const int64_t kg_tiles = Kg ? (opts->kcache_capacity + kt - 1) / kt : 0;
+    atf_repack_kernel<<<(unsigned)bq, 256, 0, s>>>((const __nv_bfloat16*)Q, Qp, rows_q, d, Nq, Nq, nullptr, 0, 0);
+    atf_repack_kernel<<<(unsigned)bk, 256, 0, s>>>((const __nv_bfloat16*)K, Kp, rows_k, d, N, kv_head_rows, Kg, kg_tiles,
+                                                   N - Nq);
     ATF_CUDA_CHECK(cudaGetLastError());
   }
 
   CUtensorMap tq, tk, tv;
-  if ((st = make_tile_map(&tq, Qp, (int64_t)B * Hq, Nq, d)) != ATF_OK) return st;
-  if ((st = make_tile_map(&tk, Kp, (int64_t)B * Hkv, N, d)) != ATF_OK) return st;
-  if ((st = make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, kv_head_rows)) != ATF_OK) return st;
+  if ((st = atf_make_tile_map(&tq, Qp, (int64_t)B * Hq, Nq, d, Nq, T)) != ATF_OK) return st;
+  if ((st = atf_make_tile_map(&tk, Kp, (int64_t)B * Hkv, N, d, N, T)) != ATF_OK) return st;
+  if ((st = atf_make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, kv_head_rows, T)) != ATF_OK) return st;
 
   PrefillParams P;
   P.sched = sched;

@@ -162,7 +162,8 @@ def _decode_case(atf, w: gen.Workload, mode, table=None):
 
 
 def test_kcache_pack_layout(atf):
-    """Tile T, group j of the packed cache hold pairs r = h-1-8j-i (i = 0..7) of keys T*KT.. as (dim r, dim r+h)."""
+    """Tile T, group j of the packed cache hold pairs r = h-1-8j-i (i = 0..7) of keys T*KT.. as (dim r, dim r+h);
+    keys whose index in the tile has bit 2 set store the two 16-byte halves of that entry swapped."""
     B, Hkv, n, d = 2, 3, 150, 128
     h, kt = d // 2, 64
     K = gen.normal_bf16((B, Hkv, n, d), 123).cuda()
@@ -174,8 +175,9 @@ def test_kcache_pack_layout(atf):
         for j in range(d // 16):
             for i in range(8):
                 r = h - 1 - (8 * j + i)
-                ref[:, :, pos // kt, j, pos % kt, 2 * i] = K[:, :, m, r]
-                ref[:, :, pos // kt, j, pos % kt, 2 * i + 1] = K[:, :, m, r + h]
+                e = 2 * i if not ((pos % kt) >> 2) & 1 else (2 * i + 8) % 16
+                ref[:, :, pos // kt, j, pos % kt, e] = K[:, :, m, r]
+                ref[:, :, pos // kt, j, pos % kt, e + 1] = K[:, :, m, r + h]
     assert torch.equal(Kg, ref)
 
 
