@@ -91,8 +91,10 @@ struct PrefillSmem {
 // B_SFULL / B_PV0 / B_OFULL / B_QZ: slot + X for query tile X (0 = A, 1 = B); B_PFULL: slot + 2 * X + h
 // for key half h of the tile.  B_PV0: the product O_X += P(half 0) V of the step is complete.
 // B_ORDER + X: issuer X has issued the closing batch of its step on the current key tile.
+// d = 64 only (P has tensor-memory columns of its own there): B_SREAD + X: every softmax warp of tile X holds
+// its part of S in registers, the next S may be written; B_PV1 + X: O_X += P(half 1) V of the step is complete.
 enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_PV0 = 11, B_PFULL = 13,
-       B_OFULL = 17, B_QZ = 19, B_ORDER = 21, B_COUNT = 23 };
+       B_OFULL = 17, B_QZ = 19, B_ORDER = 21, B_SREAD = 23, B_PV1 = 25, B_COUNT = 27 };
 constexpr int HK = T / 2;  // keys per half tile: S and P are produced and consumed in halves
 
 __global__ void __launch_bounds__(256)
@@ -270,6 +272,11 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   constexpr int H = D / 2;
   constexpr int NB = D / 64;
   constexpr uint32_t TMEM_COLS = 512;
+  // Tensor memory: S_A, S_B (128 columns each), O_A, O_B (D columns each).  At d = 128 that is all 512 columns
+  // and P (bf16) is written over the S columns it came from, so the next S has to wait for O += P V.  At
+  // d = 64 there are 128 columns left: P gets them (64 per query tile), and the next S is issued as soon as
+  // the softmax group holds the current one in registers, a whole product earlier.
+  constexpr bool FREE_P = D == 64;
   constexpr uint32_t IDESC_QK = make_idesc_bf16(128, T, 0, 0);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(128, D, 0, 1);
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
@@ -309,6 +316,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       mbar_init(bar(B_SFULL + x), 1);
       mbar_init(bar(B_PV0 + x), 1);
       mbar_init(bar(B_ORDER + x), 1);
+      mbar_init(bar(B_SREAD + x), 4);
+      mbar_init(bar(B_PV1 + x), 1);
       for (int h = 0; h < 2; ++h) mbar_init(bar(B_PFULL + 2 * x + h), 4);  // one arrival per softmax warp of the tile
       mbar_init(bar(B_OFULL + x), 1);
       mbar_init(bar(B_QZ + x), 128);
@@ -421,7 +430,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // MN-major descriptor.  `first` marks the very first product of the query tile.
       auto issue_pv = [&](int tile, int h, bool first) {
         const uint64_t v0 = ((tile & 1) ? dV1 : dV0) + (uint64_t)(h * 512);
-        const uint32_t tOx = tmem_base + 2 * T + X * D, tPx = tmem_base + X * T + h * HK;
+        const uint32_t tOx = tmem_base + 2 * T + X * D;
+        const uint32_t tPx = FREE_P ? tmem_base + 2 * T + 2 * D + X * 64 + h * 32 : tmem_base + X * T + h * HK;
         asm volatile(
             "{\n\t"
             ".reg .pred pf, pt;\n\t"
@@ -482,26 +492,36 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tc_fence_after();
         issue_pv(t, 0, v == 0);
         tc_commit(bar(B_PV0 + X));
+        if (FREE_P && more) {
+          // the softmax group has S(v) in registers: S(v + 1) can go over it while the group is still at work
+          if (!wait_or_abort(bar(B_SREAD + X), v & 1, abortp)) { ok = false; fail_site = 27; break; }
+          tc_fence_after();
+          issue_qk(t + 1, natoms);
+          tc_commit(bar(B_SFULL + X));
+        }
         if (!wait_or_abort(bar(B_PFULL + 2 * X + 1), v & 1, abortp)) { ok = false; fail_site = 23; break; }
         // The closing batches of the two query tiles go to the tensor pipe in a fixed order, tile B's
         // for key tile t, tile A's for key tile t, tile B's for t + 1, ...  Issued at the same time
         // they would interleave and both finish late, and the two softmax groups would then work and
         // wait in step with each other; one after the other, each group works while the other waits.
         // A batch is announced only where the other issuer waits for it.
-        if (ATF_ORDER_BATCHES) {
+        if (ATF_ORDER_BATCHES && !FREE_P) {
           const bool other_before = X == 0 ? t < nB : (t >= 2 && t - 1 <= nA);  // tile B's batch of t / tile A's of t - 1
           const int tp = X == 0 ? t : t - 1;                                  // its key tile: announcements start at 1
           if (other_before && !wait_or_abort(bar(B_ORDER + (X ^ 1)), (tp - 1) & 1, abortp)) { ok = false; fail_site = 26; break; }
         }
         tc_fence_after();
         issue_pv(t, 1, false);
-        if (more) {
+        if (FREE_P) {
+          tc_commit(bar(B_PV1 + X));
+          if (!more) tc_commit(bar(B_OFULL + X));
+        } else if (more) {
           issue_qk(t + 1, natoms);
           tc_commit(bar(B_SFULL + X));  // S(v + 1) is there, and every product before it is complete
         } else {
           tc_commit(bar(B_OFULL + X));
         }
-        if (ATF_ORDER_BATCHES) {
+        if (ATF_ORDER_BATCHES && !FREE_P) {
           const bool other_waits = X == 0 ? t + 1 < nB : (t >= 1 && t <= nA);
           if (other_waits) mbar_arrive(bar(B_ORDER + X));
         }
@@ -523,6 +543,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem_base + X * T + lane_off;
     const uint32_t tO = tmem_base + 2 * T + X * D + lane_off;
+    // where P(half h) goes: columns of its own at d = 64, the first 32 columns of the half's S otherwise
+    const uint32_t tP0 = FREE_P ? tmem_base + 2 * T + 2 * D + X * 64 + lane_off : tS;
+    constexpr int P_HALF_COLS = FREE_P ? 32 : HK;
     uint8_t* qrow_base = smem_gen + SM::Q_OFF + X * SM::TILE;
 
     bool ok = wait_or_abort(bar(B_QFULL), 0, abortp);
@@ -563,6 +586,8 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     // below, one step at a time.
     int t = 0;
     int h_enter = 0;  // half at which the general step starts (1: the plain loop handed over its second half)
+    bool s_released = false;  // d = 64: the half handed over is no longer in tensor memory
+    bool s_seen = false;      // the plain loop has waited for S of the step it hands over
     while (ok) {
       // ---------------- plain steps ----------------
       for (; t < Tt; ++t) {
@@ -580,19 +605,30 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
           tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
           tc_wait_ld();
+          if (FREE_P && h == 1) {  // all of S(v) is in registers now
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_SREAD + X));
+          }
           uint32_t pk[HK / 2];
           const float lsum = exp_half<POLY_OF_4>(s, kScaleLog2, -m_used * kScaleLog2, pk);
           if (__any_sync(0xffffffffu, !(lsum < STALE_REF_GUARD))) {
-            // S is still in tensor memory (P has not been stored): the general step redoes this half
+            // The general step redoes this half.  S is still in tensor memory (P has not been stored) unless
+            // its columns have just been released (d = 64, second half): then the half is recomputed from Q and K.
             h_enter = h;
             handed_over = true;
+            s_seen = true;
+            s_released = FREE_P && h == 1;
             break;
           }
           if (h == 1) {  // done with this K tile: both halves of S have been computed
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(B_KEMPTY + ks));
           }
-          tc_st32(tS + c0, pk);
+          if (FREE_P && h == 1) {  // the product that read the previous P(half 1) must be complete
+            if (!wait_or_abort(bar(B_PV1 + X), (v - 1) & 1, abortp)) { ok = false; fail_site = 38; break; }
+          }
+          tc_st32(tP0 + h * P_HALF_COLS, pk);
           l_run += lsum;
           if (h == 0) {
             if (COUNT && row_ok) {  // every cell of the tile holds the same pairs (coarse: whole groups of 8, i.e. 8 per MMA step)
@@ -637,19 +673,49 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
       }
 
-      if (!wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
+      // (not again for a step the plain loop hands over: at d = 64 the barrier may be a phase further by now)
+      if (!s_seen && !wait_or_abort(bar(B_SFULL + X), v & 1, abortp)) { ok = false; fail_site = 32; break; }
+      s_seen = false;
       tc_fence_after();
 #pragma unroll 1
       for (int h = h_enter; h < 2; ++h) {
         const int c0 = h * HK;  // first key column of this half
         float s[HK];
-        if (natoms > 0) {
-          tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
-          tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
-          tc_wait_ld();
-        } else {
+        if (FREE_P && s_released) {
+          // S(v) has been given up already: this half again from Q and K, pair by pair.  A plain step: every
+          // cell holds the same pairs (coarse mode: the tile's whole groups of 8), none of them zeroed in Q.
+          if (!wait_or_abort(bar(B_KFULL + ks), (t / KS) & 1, abortp)) { ok = false; fail_site = 31; break; }
+          const int np = MODE == ATF_MODE_EXACT ? p_all : min(H, 8 * natoms);
 #pragma unroll
           for (int c = 0; c < HK; ++c) s[c] = 0.f;
+          for (int p = 0; p < np; ++p) {
+            const uint32_t qq = *reinterpret_cast<const uint32_t*>(qsrc + 2 * p);
+            const float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
+            const int col = 2 * p;
+            const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+            const int chunk = (col & 63) >> 3;
+#pragma unroll
+            for (int c = 0; c < HK; ++c) {
+              uint32_t kk;
+              asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk) : "r"(kb32 + ((chunk ^ (c & 7)) << 4) + (c0 + c) * 128));
+              s[c] = fmaf(q0, bf16lo_to_f32(kk), fmaf(q1, bf16hi_to_f32(kk), s[c]));
+            }
+          }
+          s_released = false;
+        } else {
+          if (natoms > 0) {
+            tc_ld32(tS + c0, reinterpret_cast<uint32_t*>(s));
+            tc_ld32(tS + c0 + 32, reinterpret_cast<uint32_t*>(s) + 32);
+            tc_wait_ld();
+          } else {
+#pragma unroll
+            for (int c = 0; c < HK; ++c) s[c] = 0.f;
+          }
+          if (FREE_P && h == 1) {  // all of S(v) is in registers now
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_SREAD + X));
+          }
         }
 
         uint32_t pk[HK / 2];  // P (bf16) goes over the first 32 columns of this half of S (column c holds keys 2c, 2c+1)
@@ -744,6 +810,9 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (h == 1) {
               if (!wait_or_abort(bar(B_PV0 + X), v & 1, abortp)) { ok = false; fail_site = 34; break; }
               tc_fence_after();
+            } else if (FREE_P && v > 0) {  // d = 64: S(v) was issued before O += P(v - 1, 1) V
+              if (!wait_or_abort(bar(B_PV1 + X), (v - 1) & 1, abortp)) { ok = false; fail_site = 34; break; }
+              tc_fence_after();
             }
   #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {
@@ -763,7 +832,10 @@ atf_prefill_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           if (lane == 0) mbar_arrive(bar(B_KEMPTY + ks));
         }
 
-        tc_st32(tS + c0, pk);
+        if (FREE_P && h == 1 && v > 0) {  // the product that read the previous P(half 1) must be complete
+          if (!wait_or_abort(bar(B_PV1 + X), (v - 1) & 1, abortp)) { ok = false; fail_site = 38; break; }
+        }
+        tc_st32(tP0 + h * P_HALF_COLS, pk);
         l_run = l_run * scale_o + lsum;
 
         if (h == 0) {
