@@ -324,8 +324,10 @@ def run_ours(args):
     for k, kw in arms.items():  # warm-up of each arm
         atf.atf_prefill(Qg, Kg, V, O=O, LSE=LSE, **kw)
     torch.cuda.synchronize()
-    for _ in range(args.reps):
-        for k, kw in arms.items():
+    order = list(arms)
+    for rep in range(args.reps):
+        for k in order[rep % 3:] + order[:rep % 3]:  # rotate the order: no arm always runs behind the same one
+            kw = arms[k]
             a, b_ = ev(), ev()
             w0 = time.time()
             a.record()
@@ -492,6 +494,30 @@ def run_decode_only(args, atf, wl, pk, dev):
                       "clocks": clocks}))
 
 
+def run_probe_lines(args):
+    """What DRAM moves when parts of 256-byte rows are left out (the library's read diagnostic): one line per mask."""
+    import paper_2608_02947_b200 as atf
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    atf.ensure_workspace(1 << 20, dev)
+    buf = torch.ones(1 << 30, dtype=torch.uint8, device=dev)
+    for mask in (0xFFFF, 0xF0F0, 0xFCFC, 0xFF00, 0x00FF, 0xF000):
+        best = 1e9
+        for rep in range(6):
+            a, b_ = ev(), ev()
+            a.record()
+            atf.binding.probe_masked_read(buf, mask)
+            b_.record()
+            torch.cuda.synchronize()
+            if rep:
+                best = min(best, a.elapsed_time(b_))
+        live = bin(mask).count("1")
+        print(json.dumps({"probe_lines": True, "mask": f"{mask:04x}", "live_chunks_of_16": live, "ms": best,
+                          "requested_GB": buf.numel() * live / 16 / 1e9,
+                          "requested_GBps": buf.numel() * live / 16 / best / 1e6,
+                          "whole_rows_GBps": buf.numel() / best / 1e6}))
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -592,11 +618,15 @@ def main():
                     help="time only decode on the workload's cache shape (for the B = 8 configurations)")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only the warm-up and timed steps (for profiler captures); prints a short line")
+    ap.add_argument("--probe-lines", action="store_true",
+                    help="time the library's masked row-read diagnostic (DRAM line granularity) and exit")
     ap.add_argument("--replica-selftest", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         spawn_replicas(args)
-    if args.replica_selftest:
+    if args.probe_lines:
+        run_probe_lines(args)
+    elif args.replica_selftest:
         run_replica_selftest(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -274,6 +274,13 @@ atf_status atf_check_status_at(void* workspace, void* stream);
  * and records it in the bound workspace.  The next atf_check_status returns ATF_ERR_TIMEOUT once. */
 atf_status atf_selftest_bounded_wait(unsigned int limit_us, void* stream);
 
+/* Diagnostic behind the choice of K-cache layouts: reads `bytes` of device memory as 256-byte rows (a K row
+ * at d = 128), leaving out the 16-byte chunks of every row whose bit in chunkmask (16 bits, bit c = chunk c)
+ * is clear.  Timed by the caller; with the DRAM counters of a profiler it shows that a chunk skipped inside
+ * a 128-byte line saves no traffic (a mask like 0xF0F0 costs what 0xFFFF costs), while whole lines do
+ * (0xFF00).  Needs a bound workspace (one word of it is the kernel's sink).                              */
+atf_status atf_probe_masked_read(const void* buf, size_t bytes, unsigned int chunkmask, void* stream);
+
 /* Text of the calling thread's last error ("" if none). Never NULL. */
 const char* atf_last_error(void);
 

@@ -76,11 +76,12 @@ def lib():
     L.atf_check_status.argtypes = [vp]
     L.atf_check_status_at.argtypes = [vp, vp]
     L.atf_selftest_bounded_wait.argtypes = [C.c_uint, vp]
+    L.atf_probe_masked_read.argtypes = [vp, C.c_size_t, C.c_uint, vp]
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
                  "atf_kcache_pack",
-                 "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait"):
+                 "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait", "atf_probe_masked_read"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -425,3 +426,10 @@ def check_status(workspace=None):
 def selftest_bounded_wait(limit_us=1000):
     """Launches the library's wait-that-runs-out self-test on the current device (needs a bound workspace)."""
     _check(lib().atf_selftest_bounded_wait(int(limit_us), C.c_void_p(torch.cuda.current_stream().cuda_stream)))
+
+
+def probe_masked_read(buf, chunkmask):
+    """Launches the row-read diagnostic on a CUDA byte buffer (see atf_probe_masked_read in the header)."""
+    with torch.cuda.device(buf.device):
+        _check(lib().atf_probe_masked_read(C.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size(), int(chunkmask),
+                                           C.c_void_p(torch.cuda.current_stream(buf.device).cuda_stream)))

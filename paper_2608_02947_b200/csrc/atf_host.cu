@@ -122,6 +122,34 @@ __global__ void atf_bounded_wait_selftest_kernel(unsigned int* status, unsigned 
   }
 }
 
+// Reads a buffer as 256-byte rows (a K row at d = 128), two rows per warp instruction, lane % 16 = the 16-byte
+// chunk of the row; chunks whose bit in `chunkmask` is clear are not read.  Only the time and the DRAM
+// counters matter: it shows what leaving out parts of a row saves at DRAM's 128-byte line granularity.
+__global__ void __launch_bounds__(256) atf_probe_masked_read_kernel(const uint4* __restrict__ buf, size_t nrows,
+                                                                     unsigned chunkmask, unsigned* sink) {
+  const int lane = threadIdx.x & 31, c = lane & 15, sub = lane >> 4;
+  const bool live = (chunkmask >> c) & 1;
+  const size_t warp = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5;
+  const size_t nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
+  const size_t per_warp = (nrows + nwarps - 1) / nwarps;
+  const size_t r0 = warp * per_warp, r1 = r0 + per_warp < nrows ? r0 + per_warp : nrows;
+  unsigned acc = 0;
+  for (size_t r = r0; r + 16 <= r1; r += 16) {
+    uint4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (live)
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w)
+                     : "l"(buf + (r + 2 * i + sub) * 16 + c));
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc ^= v[i].x ^ v[i].y ^ v[i].z ^ v[i].w;
+  }
+  if (acc == 0x12345678u) sink[0] = acc;  // keeps the loads alive
+}
+
 size_t atf_decode_workspace_bytes(int B, int Hq, int Hkv, int64_t L, int d);
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d);
 
@@ -244,6 +272,15 @@ atf_status atf_check_status_at(void* workspace, void* stream) {
   atf_status rc = read_status_words(workspace, (cudaStream_t)stream, st);
   if (rc != ATF_OK) return rc;
   if (st[0] != 0) return atf_fail(ATF_ERR_TIMEOUT, "a kernel gave up a bounded wait (code %u at site %u)", st[0], st[1]);
+  return ATF_OK;
+}
+
+atf_status atf_probe_masked_read(const void* buf, size_t bytes, unsigned int chunkmask, void* stream) {
+  if (!buf || bytes < (1u << 20) || ((uintptr_t)buf & 255)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_probe_masked_read: need a 256-byte aligned buffer of at least 1 MiB");
+  if (!g_ws.ptr) return atf_fail(ATF_ERR_WORKSPACE, "atf_probe_masked_read: no workspace bound");
+  atf_probe_masked_read_kernel<<<148 * 8, 256, 0, (cudaStream_t)stream>>>((const uint4*)buf, bytes / 256, chunkmask & 0xFFFFu,
+                                                                          (unsigned*)g_ws.ptr + 16);
+  ATF_CUDA_CHECK(cudaGetLastError());
   return ATF_OK;
 }
 
