@@ -14,10 +14,15 @@ Pinned functions (pins live in tests/test_oracle_*.py, all CPU-only):
                                     pure-Python brute force
   kept_terms_*                    - printed shares (Table 1, Fig. 7), closed forms (Eq. 5,
                                     App. C), brute force
-  coarse_* (second named mode)    - the speed ceilings of Table 4 pin the rounding rule; the
-                                    numerical result of the coarse mode is otherwise defined
-                                    here only: PARITY UNPINNED for coarse_attention_rows and
-                                    coarse_decode beyond those ceilings.
+  coarse_* (second named mode)    - the speed ceilings of Table 4 pin the rounding rule of the
+                                    count; coarse_first_pair / coarse_attention_rows /
+                                    coarse_decode are tied to that count and to the per-term
+                                    definition on a raised table (tests/test_oracle_coarse_pins.py).
+                                    What stays a reading: nearest versus farthest cell of a tile
+                                    at Table 4's printed precision, and the tile size.
+  window_table_family             - Table 2's pruned shares (arithmetic and constant profiles);
+                                    the geometric profile: PARITY UNPINNED (App. A names it and
+                                    prints no value).
 """
 from __future__ import annotations
 

@@ -115,7 +115,7 @@ def test_prefill_dropped_keys_and_uniform_table(atf):
 
 
 def test_prefill_tiny_config(atf):
-    """BASELINE config 0: B=1, Hq=2, Hkv=1, d=64, base 1e6, N=2048, k=2, and k=inf = full attention."""
+    """The tiny prefill workload: B=1, Hq=2, Hkv=1, d=64, base 1e6, N=2048, k=2, and k=inf = full attention."""
     w = gen.tiny()
     O2, L2 = _prefill_case(atf, w, None, atf.ATF_MODE_EXACT)
     winf = gen.tiny(k=math.inf)
@@ -198,7 +198,7 @@ def test_decode_dropped_keys(atf):
 
 
 def test_decode_llama_32k(atf):
-    """BASELINE config 3 at B=1, L=32768 (Llama-3.2-3B shape, llama3-scaled table)."""
+    """The Llama-3.2-3B decode workload at B=1, L=32768 (llama3-scaled table)."""
     w = gen.llama32_3b(32768, B=1, seed_off=7)
     _decode_case(atf, w, 0)
     _decode_case(atf, w, 1)
