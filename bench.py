@@ -358,7 +358,8 @@ def run_ours(args):
     del Qh, Oh2
     half_exec, _ = prefill_flops(wl, Wl, n0=wl.N // 2)
 
-    dec = time_decode(atf, wl, W, Wl, qd, Kg, V, Kcache, Od)
+    _, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+    dec = time_decode(atf, wl, W, Wl, qd, Kg, V, Kcache, Od, theta)
     dbytes, dbytes_full, dfetch = dec["alg_bytes"], dec["full_bytes"], dec["fetched_bytes"]
     dec_us, dec_full_us, dec_grp_us = dec["rows_us"], dec["rows_full_us"], dec["groups_us"]
 
@@ -407,6 +408,8 @@ def run_ours(args):
         # decode on the group-major cache the prefill wrote (the pipeline's path); alone, cycling the pool
         "decode_us": dec_grp_us, "decode_gbs": dbytes / (dec_grp_us * 1e-6) / 1e9,
         "decode_speedup_vs_full": dec_full_us / dec_grp_us, "decode_in_step_us": dec_ms * 1e3,
+        # the same step on a position-independent (unrotated) cache: the kernel rotates what it fetches (App. B)
+        "decode_rotate_at_read_us": dec["groups_rot_us"],
         # decode on the row-layout cache (atf_decode's default): every K row is read whole, so the window saves no traffic
         "decode_rows_us": dec_us, "decode_rows_gbs": dbytes / (dec_us * 1e-6) / 1e9,
         "decode_full_us": dec_full_us, "decode_full_gbs": dbytes_full / (dec_full_us * 1e-6) / 1e9,
@@ -439,34 +442,38 @@ def run_ours(args):
     print(json.dumps(out))
 
 
-def time_decode(atf, wl, W, Wl, qd, Kg, V, Kcache, Od):
+def time_decode(atf, wl, W, Wl, qd, Kg, V, Kcache, Od, theta):
     """Decode alone, cycling a KV pool of >= 512 MiB so that no read hits L2 from an earlier one.  Each timed
     region holds DEC_BATCH launches back to back (one per pool entry in turn), so the device queue stays full and
-    the host's call overhead (~15 us per call through the binding) is not billed to the kernel."""
+    the host's call overhead (~15 us per call through the binding) is not billed to the kernel.
+    The "rot" arm is the rotate-at-read decode (App. B) on the same group-major bytes taken as unrotated keys: its
+    cost does not depend on the values."""
     kv_bytes = 2 * Kg.numel() * 2
     npool = max(2, math.ceil((512 << 20) / kv_bytes) + 1)
     pool = [(Kg, V)] + [(Kg.clone(), V.clone()) for _ in range(npool - 1)]
     gpool = [Kcache] + [Kcache.clone() for _ in range(npool - 1)]  # the caches the prefill wrote, group-major
     DEC_BATCH = 8
-    dec_t = {"win": [], "full": [], "grp": []}
-    for kind in ("win", "full", "grp"):
+    tabs = atf.atf_rope_tables(theta, wl.d, Kcache.shape[2] * Kcache.shape[4], device=qd.device)
+    dec_t = {"win": [], "full": [], "grp": [], "rot": []}
+    for kind in ("win", "full", "grp", "rot"):
         it = 0
         for rep in range(2 + 10):
             a, b_ = ev(), ev()
             a.record()
             for _ in range(DEC_BATCH):
                 Kc, Vc = pool[it % npool]
-                if kind == "grp":
+                if kind in ("grp", "rot"):
                     Kc = gpool[it % npool]
                 it += 1
-                atf.atf_decode(qd, Kc, Vc, table=None if kind == "full" else W, O=Od)
+                atf.atf_decode(qd, Kc, Vc, table=None if kind == "full" else W, O=Od,
+                               rope_tables=tabs if kind == "rot" else None)
             b_.record()
             torch.cuda.synchronize()
             if rep >= 2:
                 dec_t[kind].append(a.elapsed_time(b_) * 1e3 / DEC_BATCH)
     atf.binding.check_status()
     return {"rows_us": statistics.median(dec_t["win"]), "rows_full_us": statistics.median(dec_t["full"]),
-            "groups_us": statistics.median(dec_t["grp"]), "alg_bytes": decode_bytes(wl, Wl, True),
+            "groups_us": statistics.median(dec_t["grp"]), "groups_rot_us": statistics.median(dec_t["rot"]), "alg_bytes": decode_bytes(wl, Wl, True),
             "full_bytes": decode_bytes(wl, Wl, False), "fetched_bytes": decode_fetched_bytes(wl, Wl)}
 
 
@@ -474,7 +481,7 @@ def run_decode_only(args, atf, wl, pk, dev):
     """Decode configurations that have no prefill of their own (B = 8): post-RoPE caches drawn directly, the
     group-major cache written by the pack call; prints a short line (sweep files under profiles/)."""
     q, Kc, Vc = gen.decode_inputs(wl, device=dev)
-    W, _ = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+    W, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
     Wl = W.tolist()
     Wt = atf.WindowTable(W)
     atf.ensure_workspace(atf.atf_workspace_bytes(1, wl.B, wl.Hq, wl.Hkv, wl.N, wl.d), dev)
@@ -482,13 +489,13 @@ def run_decode_only(args, atf, wl, pk, dev):
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     w0 = time.time()
-    d = time_decode(atf, wl, Wt, Wl, q, Kc, Vc, Kcache, torch.empty_like(q))
+    d = time_decode(atf, wl, Wt, Wl, q, Kc, Vc, Kcache, torch.empty_like(q), theta)
     clocks = sampler.summary(w0, time.time())
     sampler.stop()
     print(json.dumps({"decode_only": True, "workload": args.workload, "B": wl.B, "L": wl.N,
                       "groups_us": d["groups_us"], "groups_gbs": d["alg_bytes"] / d["groups_us"] / 1e3,
                       "groups_frac_of_hbm": d["alg_bytes"] / d["groups_us"] / 1e3 / pk["hbm_gbs"],
-                      "rows_us": d["rows_us"], "rows_full_us": d["rows_full_us"],
+                      "rows_us": d["rows_us"], "rows_full_us": d["rows_full_us"], "groups_rot_us": d["groups_rot_us"],
                       "groups_speedup_vs_full": d["rows_full_us"] / d["groups_us"],
                       "alg_MB": d["alg_bytes"] / 1e6, "fetched_MB": d["fetched_bytes"] / 1e6, "full_MB": d["full_bytes"] / 1e6,
                       "clocks": clocks}))

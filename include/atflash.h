@@ -94,6 +94,10 @@ typedef struct {
                             the prefill wrote with no conversion pass (Sec. 7.2).               */
   int64_t kcache_capacity; /* keys the group-major cache is laid out for, >= N (its tile count fixes the
                               layout).  Decode with ATF_KLAYOUT_GROUPS reads it too: 0 = exactly L.    */
+  const void* rope_tables; /* decode with ATF_KLAYOUT_GROUPS only: dev, the tables atf_rope_tables wrote, or
+                              NULL.  If set, Kcache holds UNROTATED keys (position-independent, App. B)
+                              and the kernel rotates the pairs it fetches while it reads them.      */
+  int64_t rope_tables_capacity; /* the capacity the tables were built for, >= L                       */
 } atf_opts;
 
 /* Window table (Eq. 2, Eq. 3; effective frequencies per Sec. 3.2).  Host only, no GPU needed.
@@ -225,6 +229,25 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
 int64_t atf_kcache_tile_keys(int d);
 atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, int64_t n, int64_t Lcap,
                            int64_t pos0, int d, void* stream);
+
+/* Rotation tables for decode on an unrotated, position-independent K cache (App. B: a cache that is
+ * reused at another position stores keys before RoPE, and the rotation is applied at read; only the
+ * pairs the window keeps are fetched, so only those are rotated).
+ *   theta   : host, d/2 doubles, the effective frequencies (atf_window_table's theta_out);
+ *   pos0    : position of key 0 of the cache; capacity: keys the tables cover (>= every L used);
+ *   tables  : dev, 256-byte aligned, atf_rope_tables_bytes(d, capacity) bytes, owned by the caller.
+ * The tables hold (cos, sin) in fp32, computed in fp64: one row per key of a tile and one row per
+ * tile; the kernel adds the two angles.  They depend on (theta, pos0) only, so one build serves
+ * every decode step of a sequence.  Pass them as atf_opts.rope_tables with k_layout =
+ * ATF_KLAYOUT_GROUPS; the cache is written by atf_kcache_pack from UNROTATED key rows, q is rotated
+ * by the caller (atf_rope at position pos0 + L - 1).  The result equals decode on the rotated
+ * cache up to the fp32 rotation (a key element may differ by one bf16 unit in the last place).
+ * Errors: ATF_ERR_INVALID_ARG (null, misaligned, theta not positive and finite, bad range),
+ * ATF_ERR_UNSUPPORTED (d), ATF_ERR_WORKSPACE (buffer too small); atf_rope_tables_bytes returns 0 for
+ * a shape it does not support.                                                                  */
+size_t atf_rope_tables_bytes(int d, int64_t capacity);
+atf_status atf_rope_tables(const double* theta, int d, int64_t pos0, int64_t capacity, void* tables,
+                           size_t bytes, void* stream);
 
 /* Decode without any device allocation.  (The paper has no counterpart: this entry point exists
  * for the callers described here, not for a passage of the method.)

@@ -24,4 +24,6 @@ from .binding import (  # noqa: F401
     lib_path,
     llama3_scaling,
     new_kcache_groups,
+    atf_rope_tables,
+    RopeTables,
 )

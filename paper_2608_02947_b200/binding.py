@@ -27,7 +27,8 @@ class _Scaling(C.Structure):
 class _Opts(C.Structure):
     _fields_ = [("mode", C.c_int), ("kept_terms", C.c_void_p), ("lse", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("k_layout", C.c_int),
-                ("kcache_groups", C.c_void_p), ("kcache_capacity", C.c_int64)]
+                ("kcache_groups", C.c_void_p), ("kcache_capacity", C.c_int64),
+                ("rope_tables", C.c_void_p), ("rope_tables_capacity", C.c_int64)]
 
 
 def lib_path():
@@ -65,6 +66,9 @@ def lib():
     L.atf_decode.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
     L.atf_decode_ex.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), C.POINTER(_Opts), vp]
     L.atf_kcache_pack.argtypes = [vp, vp, i, i, i64, i64, i64, i, vp]
+    L.atf_rope_tables_bytes.argtypes = [i, i64]
+    L.atf_rope_tables_bytes.restype = C.c_size_t
+    L.atf_rope_tables.argtypes = [C.POINTER(C.c_double), i, i64, i64, vp, C.c_size_t, vp]
     L.atf_kcache_tile_keys.argtypes = [i]
     L.atf_kcache_tile_keys.restype = C.c_int64
     L.atf_decode_static.argtypes = [vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), vp]
@@ -80,7 +84,7 @@ def lib():
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
-                 "atf_kcache_pack",
+                 "atf_kcache_pack", "atf_rope_tables",
                  "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait", "atf_probe_masked_read"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -354,9 +358,36 @@ def atf_kcache_pack(K, Kg=None, pos0=0):
     return Kg
 
 
-def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=False, O=None):
+class RopeTables:
+    """The device tables of atf_rope_tables with the shape they were built for."""
+
+    def __init__(self, buf, d, pos0, capacity):
+        self.buf, self.d, self.pos0, self.capacity = buf, d, pos0, capacity
+
+
+def atf_rope_tables(theta, d, capacity, pos0=0, device="cuda"):
+    """Rotation tables for decode on an unrotated group-major K cache of up to `capacity` keys whose
+    key 0 sits at position pos0 (pass the result to atf_decode as rope_tables)."""
+    device = torch.device(device)
+    nbytes = lib().atf_rope_tables_bytes(int(d), int(capacity))
+    if nbytes == 0:
+        raise AtfError(1, f"atf_rope_tables: unsupported shape d={d}, capacity={capacity}")
+    th = torch.as_tensor(theta, dtype=torch.float64).cpu()
+    if th.numel() != d // 2:
+        raise AtfError(1, "theta must have d/2 entries")
+    arr = (C.c_double * th.numel())(*th.tolist())
+    with torch.cuda.device(device):
+        buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        _check(lib().atf_rope_tables(arr, int(d), int(pos0), int(capacity), C.c_void_p(buf.data_ptr()), nbytes,
+                                     C.c_void_p(torch.cuda.current_stream(device).cuda_stream)))
+    return RopeTables(buf, int(d), int(pos0), int(capacity))
+
+
+def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=False, O=None,
+               rope_tables=None):
     """One decode step: q [B,Hq,d] at position L-1 against Kcache/Vcache [B,Hkv,L,d] (bf16).
-    Kcache may also be a tiled group-major cache [B,Hkv,tiles,d/16,KT,16] from atf_kcache_pack."""
+    Kcache may also be a tiled group-major cache [B,Hkv,tiles,d/16,KT,16] from atf_kcache_pack; with
+    rope_tables (atf_rope_tables) that cache holds unrotated keys and the kernel rotates what it fetches."""
     on_host = not q.is_cuda
     if on_host:
         q, Kcache, Vcache = _host_roundtrip([q, Kcache, Vcache])
@@ -374,10 +405,19 @@ def atf_decode(q, Kcache, Vcache, table=None, mode=ATF_MODE_EXACT, kept_terms=No
     if O is None:
         O = torch.empty_like(q)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
-    dev = _one_device(q, Kcache, Vcache, O, kept_terms)
+    dev = _one_device(q, Kcache, Vcache, O, kept_terms, rope_tables.buf if rope_tables is not None else None)
     ensure_workspace(atf_workspace_bytes(ATF_OP_DECODE, B, Hq, Hkv, L, d), q.device)
     tab, _keep = _table_ptr(table, d)
     o = _opts(mode, kept_terms, lse, k_layout, kcache_groups=Kcache if k_layout == ATF_KLAYOUT_GROUPS else None)
+    if rope_tables is not None:
+        if on_host:
+            raise AtfError(1, "rope_tables need device tensors")
+        if k_layout != ATF_KLAYOUT_GROUPS:
+            raise AtfError(2, "rope_tables need a group-major K cache")
+        if rope_tables.d != d:
+            raise AtfError(1, "rope_tables were built for another head dimension")
+        o.rope_tables = rope_tables.buf.data_ptr()
+        o.rope_tables_capacity = rope_tables.capacity
     with dev:
         _check(lib().atf_decode_ex(C.c_void_p(q.data_ptr()), C.c_void_p(Kcache.data_ptr()), C.c_void_p(Vcache.data_ptr()),
                                    C.c_void_p(O.data_ptr()), B, Hq, Hkv, L, d, tab,

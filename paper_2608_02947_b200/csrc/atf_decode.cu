@@ -23,6 +23,7 @@
 // log-sum-exp and writes O (and LSE).
 #include <algorithm>
 #include <cfloat>
+#include <cmath>
 #include <cstring>
 
 #include "atf_common.cuh"
@@ -58,6 +59,8 @@ struct DecodeParams {
   unsigned long long* kept;  // may be null
   int Hq, Hkv, G, L, nsplit;
   int ktiles;                // group-major K cache: tiles per (batch, KV head), >= ceil(L / tile keys)
+  const float2* rot_key;     // unrotated cache only: (cos, sin) of key-in-tile * theta, [pair][key in tile]
+  const float2* rot_tile;    // unrotated cache only: (cos, sin) of (pos0 + tile * tile keys) * theta, [tile][pair]
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -473,9 +476,26 @@ constexpr int TL_STAGES = ATF_TL_STAGES;
 constexpr int TL_THREADS = (DEC_WARPS + 1) * 32;
 constexpr int TL_TILE_BYTES = 16384;
 constexpr int TL_STAGE_BYTES = 2 * TL_TILE_BYTES;
+#ifndef ATF_ROT_BATCH
+#define ATF_ROT_BATCH 2
+#endif
+constexpr int TL_ROT_BYTES = 1024;  // room for one row of the tile-level rotation table (keeps the stages 1 KiB aligned)
 constexpr int TL_SMEM = TL_STAGES * TL_STAGE_BYTES + 1024 /* alignment slack */ + 64 /* barriers */;
+__device__ __forceinline__ float2 lds_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
 
-template <int D, int MODE, bool COUNT>
+// One (dim r, dim r + h) pair of an unrotated key, turned by the angle a + b given as (cos, sin) of a and of b
+// (App. B: the rotation applied when the cache is read).  fp32, one rounding to bf16.
+__device__ __forceinline__ uint32_t rotate_pair(uint32_t v, float2 a, float2 b) {
+  const float c = fmaf(a.x, b.x, -a.y * b.y), s = fmaf(a.y, b.x, a.x * b.y);
+  const float x = __uint_as_float(v << 16), y = __uint_as_float(v & 0xffff0000u);
+  return pack_bf16x2(fmaf(x, c, -y * s), fmaf(y, c, x * s));
+}
+
+template <int D, int MODE, bool COUNT, bool ROT>
 __global__ void __launch_bounds__(TL_THREADS, ATF_DECODE_SLOTS_GROUPS / 148)
 atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ DecodeParams P,
                         const __grid_constant__ AtfTable table) {
@@ -488,6 +508,8 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
   constexpr int NVB = D / 64;                   // 64-column boxes of a V tile
   constexpr int PSTRIDE = D + 2;
   constexpr int GBYTES = KT * 32;               // one group of a K tile
+  // rotate-at-read: the tile's row of the tile-level (cos, sin) table rides along in the stage
+  constexpr int STAGE = TL_STAGE_BYTES + (ROT ? TL_ROT_BYTES : 0);
   const float kScaleLog2 = 1.4426950408889634f / sqrtf((float)D);
 
   extern __shared__ uint8_t dsm_raw[];
@@ -496,7 +518,7 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
   __shared__ int s_abort;
   const uint32_t sbase = (smem_u32(dsm_raw) + 1023u) & ~1023u;
   uint8_t* sgen = dsm_raw + (sbase - smem_u32(dsm_raw));
-  const uint32_t bars = sbase + TL_STAGES * TL_STAGE_BYTES;
+  const uint32_t bars = sbase + TL_STAGES * STAGE;
   auto full_bar = [&](int st) { return bars + 8u * (uint32_t)st; };
   auto empty_bar = [&](int st) { return bars + 8u * (uint32_t)(TL_STAGES + st); };
 
@@ -564,9 +586,10 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
         while (r_near > 0 && sW[r_near - 1] >= z_near) --r_near;
         const int rq = MODE == ATF_MODE_COARSE ? (r_near & ~7) : r_near;
         const int ngl = (H - rq + 7) >> 3;  // live groups of the nearest key: the prefix to fetch
-        const uint32_t kdst = sbase + st * TL_STAGE_BYTES, vdst = kdst + TL_TILE_BYTES;
-        mbar_expect_tx(full_bar(st), (uint32_t)(ngl * GBYTES + TL_TILE_BYTES));
+        const uint32_t kdst = sbase + st * STAGE, vdst = kdst + TL_TILE_BYTES;
+        mbar_expect_tx(full_bar(st), (uint32_t)(ngl * GBYTES + TL_TILE_BYTES + (ROT ? ngl * 64 : 0)));
         bulk_load_1d(kdst, Kb + (int64_t)t * KT * D, (uint32_t)(ngl * GBYTES), full_bar(st));
+        if (ROT) bulk_load_1d(kdst + TL_STAGE_BYTES, P.rot_tile + (int64_t)t * H, (uint32_t)(ngl * 64), full_bar(st));
 #pragma unroll
         for (int vb = 0; vb < NVB; ++vb)
           tma_load_3d(vdst + vb * (KT * 128), &tmV, full_bar(st), vb * 64, t * KT, (int)grp);
@@ -603,7 +626,7 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
     for (int t = t_first; t < ntiles; t += P.nsplit, ++it) {
       const int st = it % TL_STAGES;
       if (!bounded_wait(full_bar(st), (it / TL_STAGES) & 1)) { fail_site = 41; break; }
-      const uint32_t ks = sbase + st * TL_STAGE_BYTES, vs = ks + TL_TILE_BYTES;
+      const uint32_t ks = sbase + st * STAGE, vs = ks + TL_TILE_BYTES;
       const int kb0 = t * KT + warp * KB;
       const bool blk_fast = (kb0 + KB <= L) && (L - 1 - kb0 <= Wmax);
 
@@ -635,21 +658,49 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
 
       // ---- S = q K^T: K step j = the 8 pairs of group j; a key with first live pair r keeps its first H - r pairs ----
       const int ngl = (H - rq_near + 7) >> 3;
+      // Rotate-at-read works on JB groups per branch, so that the table reads and the rotations of several
+      // groups overlap; a group beyond the fetched prefix holds stale bytes, which the masks below zero.
+      constexpr int JB = ROT ? ATF_ROT_BATCH : 1;
 #pragma unroll
-      for (int j = 0; j < NKS; ++j) {
-        if (j >= ngl) continue;  // warp-uniform
+      for (int jb = 0; jb < NKS; jb += JB) {
+        if (jb >= ngl) continue;  // warp-uniform
+        float2 ak[ROT ? JB : 1][ROT ? NKG / 2 : 1][2][2], at[ROT ? JB : 1][2];
+        if (ROT) {
 #pragma unroll
-        for (int kp = 0; kp < NKG / 2; ++kp) {
-          uint32_t bf[4];
-          ldsm_x4(ks + j * GBYTES + kp * 512 + k_lane_off, bf);
+          for (int jj = 0; jj < JB; ++jj)
 #pragma unroll
-          for (int h2 = 0; h2 < 2; ++h2) {
-            const int live = H - r_lane[2 * kp + h2];
-            if (8 * j + t4 >= live) bf[2 * h2] = 0u;
-            if (8 * j + 4 + t4 >= live) bf[2 * h2 + 1] = 0u;
+            for (int c = 0; c < 2; ++c) {
+              const int p = 8 * (jb + jj) + 4 * c + t4;
+              at[jj][c] = lds_f2(ks + TL_STAGE_BYTES + p * 8);
+#pragma unroll
+              for (int kp = 0; kp < NKG / 2; ++kp)
+#pragma unroll
+                for (int h2 = 0; h2 < 2; ++h2) ak[jj][kp][c][h2] = __ldg(P.rot_key + p * KT + warp * KB + (2 * kp + h2) * 8 + g);
+            }
+        }
+#pragma unroll
+        for (int jj = 0; jj < JB; ++jj) {
+          const int j = jb + jj;
+#pragma unroll
+          for (int kp = 0; kp < NKG / 2; ++kp) {
+            uint32_t bf[4];
+            ldsm_x4(ks + j * GBYTES + kp * 512 + k_lane_off, bf);
+            if (ROT) {
+              // bf[2 * h2 + c] is pair 8j + 4c + t4 of key (2kp + h2) * 8 + g of the warp's part of the tile
+#pragma unroll
+              for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int h2 = 0; h2 < 2; ++h2) bf[2 * h2 + c] = rotate_pair(bf[2 * h2 + c], at[jj][c], ak[jj][kp][c][h2]);
+            }
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const int live = H - r_lane[2 * kp + h2];
+              if (8 * j + t4 >= live) bf[2 * h2] = 0u;
+              if (8 * j + 4 + t4 >= live) bf[2 * h2 + 1] = 0u;
+            }
+            mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
+            mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
           }
-          mma_bf16_16816(sc[2 * kp], qa[j][0], qa[j][1], bf[0], bf[1]);
-          mma_bf16_16816(sc[2 * kp + 1], qa[j][0], qa[j][1], bf[2], bf[3]);
         }
       }
       if (COUNT && t4 == 0) {
@@ -869,11 +920,13 @@ atf_status launch_decode_tiles(const CUtensorMap& tmV, const DecodeParams& P, co
   dim3 grid(P.nsplit, P.Hkv, B);
 #define ATF_TL_LAUNCH(MODE_, COUNT_)                                                                        \
   do {                                                                                                      \
-    auto kern = atf_decode_tiles_kernel<D, MODE_, COUNT_>;                                                  \
-    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TL_SMEM));       \
+    auto kern = P.rot_tile ? atf_decode_tiles_kernel<D, MODE_, COUNT_, true>                                \
+                           : atf_decode_tiles_kernel<D, MODE_, COUNT_, false>;                              \
+    const int smem = TL_SMEM + (P.rot_tile ? TL_STAGES * TL_ROT_BYTES : 0);                                 \
+    ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));          \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,               \
                                         cudaSharedmemCarveoutMaxShared));                                    \
-    kern<<<grid, TL_THREADS, TL_SMEM, s>>>(tmV, P, t);                                                      \
+    kern<<<grid, TL_THREADS, smem, s>>>(tmV, P, t);                                                           \
   } while (0)
   if (mode == ATF_MODE_EXACT) {
     if (count) ATF_TL_LAUNCH(ATF_MODE_EXACT, true); else ATF_TL_LAUNCH(ATF_MODE_EXACT, false);
@@ -944,6 +997,19 @@ extern "C" atf_status atf_decode_ex(const void* q, const void* Kcache, const voi
   const int64_t cap = (opts && opts->kcache_capacity > 0) ? opts->kcache_capacity : L;
   if (cap < L) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: kcache_capacity (%lld) is smaller than L", (long long)cap);
   P.ktiles = (int)((cap + kt - 1) / kt);
+  P.rot_tile = nullptr;
+  P.rot_key = nullptr;
+  if (opts && opts->rope_tables) {
+    // App. B: the cache holds position-independent (unrotated) keys and the rotation happens at read
+    if (kl_ != ATF_KLAYOUT_GROUPS)
+      return atf_fail(ATF_ERR_UNSUPPORTED, "atf_decode: rope_tables needs the group-major K cache");
+    if ((uintptr_t)opts->rope_tables & 255)
+      return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: rope_tables must be 256-byte aligned");
+    const int64_t tcap = opts->rope_tables_capacity;
+    if (tcap < L) return atf_fail(ATF_ERR_INVALID_ARG, "atf_decode: rope_tables cover %lld keys, L is %lld", (long long)tcap, (long long)L);
+    P.rot_key = (const float2*)opts->rope_tables;
+    P.rot_tile = P.rot_key + kt * (d / 2);
+  }
   char* base = (char*)ws.ptr;
   P.status = (unsigned int*)base;
   P.counters = (unsigned int*)(base + ATF_WS_STATUS_BYTES);
@@ -974,6 +1040,64 @@ extern "C" atf_status atf_kcache_pack(const void* K, void* Kg, int B, int Hkv, i
   const int64_t kt = atf_kcache_tile_keys(d);
   atf_kcache_pack_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
       (const __nv_bfloat16*)K, (__nv_bfloat16*)Kg, (int64_t)B * Hkv, n, (Lcap + kt - 1) / kt, pos0, d);
+  ATF_CUDA_CHECK(cudaGetLastError());
+  return ATF_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Rotation tables for the decode on an unrotated K cache (App. B).  The angle of key m in pair r is
+// (pos0 + m) * theta_r = (pos0 + tile * KT) * theta_r + (m mod KT) * theta_r, so two small tables of
+// (cos, sin) - one row per tile, one row per key of a tile - give every angle by one angle addition.
+// Entries are computed in fp64 and stored in fp32; pairs are counted from the lowest frequency, like
+// the groups of the cache.  Layout: [pair][key in tile] then [tile][pair].
+// ------------------------------------------------------------------------------------------
+struct RotTheta {
+  double t[ATF_MAX_PAIRS];
+};
+__global__ void atf_rope_tables_kernel(const __grid_constant__ RotTheta th, long long pos0, int KT, int H, int64_t ntiles,
+                                       float2* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t nkey = (int64_t)KT * H;
+  if (i >= nkey + ntiles * H) return;
+  int p;
+  double pos;
+  if (i < nkey) {
+    p = (int)(i / KT);
+    pos = (double)(i % KT);
+  } else {
+    const int64_t k = i - nkey;
+    p = (int)(k % H);
+    pos = (double)(pos0 + (k / H) * KT);
+  }
+  double sn, cs;
+  sincos(pos * th.t[H - 1 - p], &sn, &cs);
+  out[i] = make_float2((float)cs, (float)sn);
+}
+
+extern "C" size_t atf_rope_tables_bytes(int d, int64_t capacity) {
+  if ((d != 64 && d != 128) || capacity < 1) return 0;
+  const int64_t kt = atf_kcache_tile_keys(d);
+  return (size_t)(kt + (capacity + kt - 1) / kt) * (d / 2) * sizeof(float2);
+}
+
+extern "C" atf_status atf_rope_tables(const double* theta, int d, int64_t pos0, int64_t capacity, void* tables,
+                                      size_t bytes, void* stream) {
+  if (!theta || !tables) return atf_fail(ATF_ERR_INVALID_ARG, "atf_rope_tables: null pointer");
+  if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_rope_tables: d must be 64 or 128 (got %d)", d);
+  if (capacity < 1 || pos0 < 0 || pos0 + capacity >= (1ll << 40)) return atf_fail(ATF_ERR_INVALID_ARG, "atf_rope_tables: bad range");
+  if ((uintptr_t)tables & 255) return atf_fail(ATF_ERR_INVALID_ARG, "atf_rope_tables: tables must be 256-byte aligned");
+  const size_t need = atf_rope_tables_bytes(d, capacity);
+  if (bytes < need) return atf_fail(ATF_ERR_WORKSPACE, "atf_rope_tables: buffer has %zu bytes, needs %zu", bytes, need);
+  RotTheta th;
+  for (int r = 0; r < d / 2; ++r) {
+    if (!(theta[r] > 0.0) || !std::isfinite(theta[r])) return atf_fail(ATF_ERR_INVALID_ARG, "atf_rope_tables: theta[%d] must be positive and finite", r);
+    th.t[r] = theta[r];
+  }
+  const int64_t kt = atf_kcache_tile_keys(d);
+  const int64_t ntiles = (capacity + kt - 1) / kt;
+  const int64_t total = (kt + ntiles) * (d / 2);
+  atf_rope_tables_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(th, (long long)pos0, (int)kt, d / 2,
+                                                                                              ntiles, (float2*)tables);
   ATF_CUDA_CHECK(cudaGetLastError());
   return ATF_OK;
 }
