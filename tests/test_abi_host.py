@@ -149,3 +149,20 @@ def test_family_validation_and_non_monotone_tables(atf):
     fake = C.c_void_p(4096)
     tab = (C.c_int64 * 32)(*W.tolist())
     assert lib.atf_prefill(fake, fake, fake, fake, None, 1, 2, 1, 1 << 20, 64, tab, 1, None) == 2
+
+
+def test_rope_tables_validation_without_a_device(atf):
+    lib = atf.lib()
+    th = (C.c_double * 64)(*([0.5] * 64))
+    fake = C.c_void_p(4096)
+    assert lib.atf_rope_tables_bytes(128, 131072) == (64 + 2048) * 64 * 8    # one row per key of a tile + one per tile
+    assert lib.atf_rope_tables_bytes(64, 1) == (128 + 1) * 32 * 8
+    assert lib.atf_rope_tables_bytes(96, 1024) == 0
+    assert lib.atf_rope_tables(None, 128, 0, 1024, fake, 1 << 20, None) == 1          # null theta
+    assert lib.atf_rope_tables(th, 96, 0, 1024, fake, 1 << 20, None) == 2             # d
+    assert lib.atf_rope_tables(th, 128, -1, 1024, fake, 1 << 20, None) == 1           # negative position
+    assert lib.atf_rope_tables(th, 128, 0, 1024, C.c_void_p(4100), 1 << 20, None) == 1  # misaligned
+    assert lib.atf_rope_tables(th, 128, 0, 1024, fake, 1024, None) == 4               # buffer too small
+    assert b"needs" in lib.atf_last_error()
+    th[7] = 0.0
+    assert lib.atf_rope_tables(th, 128, 0, 1024, fake, 1 << 20, None) == 1            # theta must be positive
