@@ -64,6 +64,25 @@ def normal_bf16(shape, seed, device="cpu"):
     return torch.randn(shape, generator=g, dtype=torch.float32, device=device).to(torch.bfloat16)
 
 
+def normal_f32(shape, seed, device="cpu"):
+    """i.i.d. N(0,1) in fp32 with the given seed (the same draws normal_bf16 rounds)."""
+    g = _gen(device, seed)
+    return torch.randn(shape, generator=g, dtype=torch.float32, device=device)
+
+
+def prefill_inputs_f32(w: Workload, device="cpu"):
+    """Un-rotated Q, K in fp32 and V in bf16 for the split-precision prefill (same seeds as prefill_inputs)."""
+    Q = normal_f32((w.B, w.Hq, w.N, w.d), w.seed * 3 + 0, device)
+    K = normal_f32((w.B, w.Hkv, w.N, w.d), w.seed * 3 + 1, device)
+    V = normal_bf16((w.B, w.Hkv, w.N, w.d), w.seed * 3 + 2, device)
+    if w.outlier:
+        h = w.d // 2
+        for t in (Q, K):
+            t[..., h - 4:h] *= 8
+            t[..., w.d - 4:w.d] *= 8
+    return Q, K, V
+
+
 def prefill_inputs(w: Workload, device="cpu"):
     """Un-rotated Q [B,Hq,N,d], K, V [B,Hkv,N,d] in bf16.  RoPE is applied by the caller."""
     Q = normal_bf16((w.B, w.Hq, w.N, w.d), w.seed * 3 + 0, device)

@@ -219,6 +219,29 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
                          int Hq, int Hkv, int64_t L, int d, const int64_t* table,
                          const atf_opts* opts, void* stream);
 
+/* Prefill with scores of more than bf16 input precision (App. D, "Precision as the other side of the
+ * compute-accuracy trade": a low-precision product split in two to recover accuracy, paid for with part
+ * of what the window saves; Sec. 6.2 scored five tasks with fp32 attention scores because bf16 rounding
+ * flipped low-margin retrievals under the window).
+ *   Q : dev fp32 [B, Hq, N, d], K: dev fp32 [B, Hkv, N, d], already rotated (atf_rope_f32) and never
+ *       rounded to bf16; V: dev bf16 [B, Hkv, N, d]; O: dev bf16 [B, Hq, N, d]; LSE: dev fp32
+ *       [B, Hq, N] or NULL.  All 16-byte aligned, row-major, caller-owned.
+ *   The library writes each of Q and K as hi = bf16(x) and lo = bf16(x - hi) (hi + lo holds x to 2^-17 of
+ *   its size) and accumulates S = Q_hi K_hi^T + Q_hi K_lo^T + Q_lo K_hi^T in fp32 over the live pairs of
+ *   each tile: three tensor-core products instead of one.  The window rule, both modes, the term counts
+ *   (opts->kept_terms) and the treatment of V, P and O are those of atf_prefill; every exponential is the
+ *   hardware ex2.  Against the per-term definition on the fp32 inputs the LSE is good to about
+ *   1.5e-5 x max(1, largest |logit|): a logit is a sum of products each held to ~2^-16 of its size.
+ *   opts: mode, kept_terms, workspace are read; kcache_groups and rope_tables return ATF_ERR_UNSUPPORTED.
+ *   Needs a workspace of atf_workspace_bytes(ATF_OP_PREFILL_SPLIT, ...) (the four bf16 parts).
+ *   Errors: as atf_prefill.  d = 64 or 128; causal must be 1.
+ * atf_rope_f32: atf_rope on fp32 rows, the result kept in fp32 (the fp64 rotation rounded once).      */
+atf_status atf_prefill_split(const float* Q, const float* K, const void* V, void* O, float* LSE, int B,
+                             int Hq, int Hkv, int64_t N, int d, const int64_t* table, int causal,
+                             const atf_opts* opts, void* stream);
+atf_status atf_rope_f32(float* X, int B, int H, int64_t N, int d, const double* theta, int64_t pos0,
+                        void* stream);
+
 /* Copies n rotated key rows into a group-major K cache (see ATF_KLAYOUT_GROUPS: the layout in
  * which the memory side of the window, Sec. 3.3, holds at DRAM line granularity).
  *   K : dev bf16 [B, Hkv, n, d], rows for positions pos0 .. pos0+n-1;
@@ -279,7 +302,7 @@ atf_status atf_decode_static(const void* q, const void* Kcache, const void* Vcac
  * serves prefill and decode in turn: its first 64.25 KiB (status words and decode's split
  * counters, which the kernels leave zeroed) are never used as scratch.  One call at a time may use a given
  * workspace; calls that overlap on the GPU need separate workspaces (atf_opts.workspace).     */
-enum { ATF_OP_PREFILL = 0, ATF_OP_DECODE = 1 };
+enum { ATF_OP_PREFILL = 0, ATF_OP_DECODE = 1, ATF_OP_PREFILL_SPLIT = 2 };
 size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d);
 atf_status atf_bind_workspace(void* dev_ptr, size_t bytes);
 

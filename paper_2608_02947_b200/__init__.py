@@ -24,6 +24,9 @@ from .binding import (  # noqa: F401
     lib_path,
     llama3_scaling,
     new_kcache_groups,
+    atf_prefill_split,
+    atf_rope_f32,
+    ATF_OP_PREFILL_SPLIT,
     atf_rope_tables,
     RopeTables,
 )

@@ -9,7 +9,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 ATF_MODE_EXACT, ATF_MODE_COARSE = 0, 1
-ATF_OP_PREFILL, ATF_OP_DECODE = 0, 1
+ATF_OP_PREFILL, ATF_OP_DECODE, ATF_OP_PREFILL_SPLIT = 0, 1, 2
 ATF_KLAYOUT_ROWS, ATF_KLAYOUT_GROUPS = 0, 1
 
 
@@ -55,6 +55,8 @@ def lib():
                                           C.POINTER(C.c_double)]
     L.atf_rope.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
     L.atf_prefill.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, vp]
+    L.atf_prefill_split.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
+    L.atf_rope_f32.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
     L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
     L.atf_prefill_chunk.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_chunk_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i,
@@ -84,7 +86,7 @@ def lib():
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
-                 "atf_kcache_pack", "atf_rope_tables",
+                 "atf_kcache_pack", "atf_rope_tables", "atf_prefill_split", "atf_rope_f32",
                  "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait", "atf_probe_masked_read"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -297,6 +299,51 @@ def atf_prefill(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_term
                                               C.byref(o) if o is not None else None, _stream(Q)))
     if on_host:
         return _to_pinned_host(O, O_host), (_to_pinned_host(LSE, LSE_host) if LSE is not None else None)
+    return O, LSE
+
+
+def _dev_f32(t, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise AtfError(1, f"{name} must be a contiguous CUDA fp32 tensor")
+
+
+def atf_rope_f32(X, theta, pos0=0):
+    """In-place half-split RoPE of X [B,H,N,d] (CUDA fp32) at positions pos0..pos0+N-1, kept in fp32."""
+    _dev_f32(X, "X")
+    B, H, N, d = X.shape
+    th = torch.as_tensor(theta, dtype=torch.float64).cpu()
+    arr = (C.c_double * th.numel())(*th.tolist())
+    with torch.cuda.device(X.device):
+        _check(lib().atf_rope_f32(C.c_void_p(X.data_ptr()), B, H, N, d, arr, int(pos0), _stream(X)))
+    return X
+
+
+def atf_prefill_split(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kept_terms=None, return_lse=True,
+                      O=None, LSE=None):
+    """atf_prefill with split-precision scores: Q [B,Hq,N,d] and K [B,Hkv,N,d] are CUDA fp32 (rotated, never
+    rounded to bf16), V is bf16; each score is three bf16 tensor-core products (hi*hi + hi*lo + lo*hi).
+    Returns (O bf16, LSE fp32 or None)."""
+    _dev_f32(Q, "Q")
+    _dev_f32(K, "K")
+    _dev_bf16(V, "V")
+    B, Hq, N, d = Q.shape
+    Hkv = K.shape[1]
+    if K.shape != (B, Hkv, N, d) or V.shape != K.shape:
+        raise AtfError(1, "K and V must be [B,Hkv,N,d] matching Q")
+    if O is None:
+        O = torch.empty(Q.shape, dtype=torch.bfloat16, device=Q.device)
+    _dev_bf16(O, "O")
+    if LSE is None and return_lse:
+        LSE = torch.empty((B, Hq, N), dtype=torch.float32, device=Q.device)
+    dev = _one_device(Q, K, V, O, LSE, kept_terms)
+    ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL_SPLIT, B, Hq, Hkv, N, d), Q.device)
+    tab, _keep = _table_ptr(table, d)
+    o = _opts(mode, kept_terms, None)
+    with dev:
+        _check(lib().atf_prefill_split(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                       C.c_void_p(O.data_ptr()), C.c_void_p(LSE.data_ptr()) if LSE is not None else None,
+                                       B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+                                       C.byref(o) if o is not None else None, _stream(Q)))
     return O, LSE
 
 

@@ -18,7 +18,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libatflash.so")
-SOURCES = ["atf_host.cu", "atf_rope.cu", "atf_decode.cu", "atf_prefill.cu", "atf_prefill_host.cu"]
+SOURCES = ["atf_host.cu", "atf_rope.cu", "atf_decode.cu", "atf_prefill.cu", "atf_prefill_host.cu", "atf_prefill_split.cu"]
 HEADERS = [os.path.join(CSRC, "atf_common.cuh"), os.path.join(ROOT, "include", "atflash.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 EXTRA = os.environ.get("ATF_NVCC_EXTRA", "").split()

@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(256) atf_probe_masked_read_kernel(const uint4*
 
 size_t atf_decode_workspace_bytes(int B, int Hq, int Hkv, int64_t L, int d);
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d);
+size_t atf_prefill_split_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d);
 
 extern "C" {
 
@@ -159,6 +160,7 @@ size_t atf_workspace_bytes(int op, int B, int Hq, int Hkv, int64_t N, int d) {
   if (B < 1 || Hq < 1 || Hkv < 1 || N < 1 || (d != 64 && d != 128)) return 0;
   if (op == ATF_OP_PREFILL) return atf_prefill_workspace_bytes(B, Hq, Hkv, N, d);
   if (op == ATF_OP_DECODE) return atf_decode_workspace_bytes(B, Hq, Hkv, N, d);
+  if (op == ATF_OP_PREFILL_SPLIT) return atf_prefill_split_workspace_bytes(B, Hq, Hkv, N, d);
   return 0;
 }
 
