@@ -238,6 +238,8 @@ def run_ours(args):
     pk = peaks()
     if args.decode_only:
         return run_decode_only(args, atf, wl, pk, dev)
+    if args.split_precision:
+        return run_split_precision(args, atf, wl, dev)
     Q0, K0, V = gen.prefill_inputs(wl, device=dev)  # un-rotated, on the device
     Qg, Kg = Q0.clone(), K0.clone()
     O = torch.empty_like(Qg)
@@ -501,6 +503,50 @@ def run_decode_only(args, atf, wl, pk, dev):
                       "clocks": clocks}))
 
 
+def run_split_precision(args, atf, wl, dev):
+    """Cost of the split-precision prefill (fp32 Q/K, three tensor-core products per score step) beside the bf16
+    path on the same rotated values; prints a short line (sweep file under profiles/)."""
+    W, theta = atf.atf_window_table(wl.base, wl.d, wl.k, wl.N, wl.scaling)
+    Wt = atf.WindowTable(W)
+    Q, K, V = gen.prefill_inputs_f32(wl, device=dev)
+    atf.atf_rope_f32(Q, theta)
+    atf.atf_rope_f32(K, theta)
+    Qb, Kb = Q.to(torch.bfloat16), K.to(torch.bfloat16)
+    O = torch.empty(Q.shape, dtype=torch.bfloat16, device=dev)
+    LSE = torch.empty(Q.shape[:3], dtype=torch.float32, device=dev)
+    atf.ensure_workspace(atf.atf_workspace_bytes(atf.ATF_OP_PREFILL_SPLIT, wl.B, wl.Hq, wl.Hkv, wl.N, wl.d), dev)
+    arms = {"split_exact_ms": lambda: atf.atf_prefill_split(Q, K, V, table=Wt, O=O, LSE=LSE),
+            "split_coarse_ms": lambda: atf.atf_prefill_split(Q, K, V, table=Wt, O=O, LSE=LSE, mode=atf.ATF_MODE_COARSE),
+            "split_full_ms": lambda: atf.atf_prefill_split(Q, K, V, table=None, O=O, LSE=LSE),
+            "bf16_exact_ms": lambda: atf.atf_prefill(Qb, Kb, V, table=Wt, O=O, LSE=LSE),
+            "bf16_coarse_ms": lambda: atf.atf_prefill(Qb, Kb, V, table=Wt, O=O, LSE=LSE, mode=atf.ATF_MODE_COARSE),
+            "bf16_full_ms": lambda: atf.atf_prefill(Qb, Kb, V, table=None, O=O, LSE=LSE)}
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    w0 = time.time()
+    ts = {k: [] for k in arms}
+    for rep in range(2 + 5):        # interleaved, inputs larger than L2 at the sizes this is quoted on
+        for k, fn in arms.items():
+            a, b_ = ev(), ev()
+            a.record()
+            fn()
+            b_.record()
+            torch.cuda.synchronize()
+            if rep >= 2:
+                ts[k].append(a.elapsed_time(b_))
+    clocks = sampler.summary(w0, time.time())
+    sampler.stop()
+    atf.binding.check_status()
+    out = {"split_precision": True, "workload": args.workload, "N": wl.N}
+    out.update({k: statistics.median(v) for k, v in ts.items()})
+    out["split_over_bf16_exact"] = out["split_exact_ms"] / out["bf16_exact_ms"]
+    out["split_over_bf16_coarse"] = out["split_coarse_ms"] / out["bf16_coarse_ms"]
+    out["split_window_speedup_exact"] = out["split_full_ms"] / out["split_exact_ms"]
+    out["split_window_speedup_coarse"] = out["split_full_ms"] / out["split_coarse_ms"]
+    out["clocks"] = clocks
+    print(json.dumps(out))
+
+
 def run_probe_lines(args):
     """What DRAM moves when parts of 256-byte rows are left out (the library's read diagnostic): one line per mask."""
     import paper_2608_02947_b200 as atf
@@ -623,6 +669,8 @@ def main():
                     help="run the step with table = NULL (the library's own k = infinity mode)")
     ap.add_argument("--decode-only", action="store_true",
                     help="time only decode on the workload's cache shape (for the B = 8 configurations)")
+    ap.add_argument("--split-precision", action="store_true",
+                    help="time the split-precision prefill beside the bf16 path on the workload's shape")
     ap.add_argument("--profile-only", action="store_true",
                     help="run only the warm-up and timed steps (for profiler captures); prints a short line")
     ap.add_argument("--probe-lines", action="store_true",

@@ -20,6 +20,9 @@ Pinned functions (pins live in tests/test_oracle_*.py, all CPU-only):
                                     definition on a raised table (tests/test_oracle_coarse_pins.py).
                                     What stays a reading: nearest versus farthest cell of a tile
                                     at Table 4's printed precision, and the tile size.
+  split-precision scores          - no function of their own: the reference is attention_rows on fp32 values
+                                    widened exactly; tests/test_oracle_split_precision.py derives the
+                                    tolerance from it (hi + lo representation, dropped lo x lo terms)
   window_table_family             - Table 2's pruned shares (arithmetic and constant profiles);
                                     the geometric profile: PARITY UNPINNED (App. A names it and
                                     prints no value).

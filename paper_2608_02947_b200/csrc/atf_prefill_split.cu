@@ -22,13 +22,15 @@
 //   warp 1      MMA issuer (one thread)
 //   warps 4-7   softmax, one query row per thread: read S, finish the window rule per cell,
 //               mask, online softmax with lazy rescaling of O, write P (bf16) to tensor memory
-// Exact mode: the MMA depth of a tile is the pairs live in ANY of its cells, rounded up to a
-// 16-column step; the pairs of that last step that are live nowhere are zeroed in the CTA's
-// copies of Q_hi and Q_lo (pairs only die as the distance grows, the tiles are walked outwards
-// from the diagonal, so the zeroing is monotone); pairs live in some cells and dead in others
-// ("straddling") are taken back out of the dead cells on the CUDA cores with the same three
-// products.  Coarse mode: depth = pairs live anywhere in the tile rounded up to 8, every pair on
-// the diagonal tile, no per-cell work.  Term counts are those of atf_prefill, bit for bit.
+// Exact mode, per quarter of the query rows (one softmax warp) as in atf_prefill: pairs live in every
+// cell of the quarter's 32 x 128 cells need nothing; a pair live in most of them stays in the MMA
+// and its three products are taken back out of the cells beyond its window on the CUDA cores; a
+// pair live in a minority is zeroed in the quarter's rows of the CTA's copies of Q_hi and Q_lo and
+// added where it is live (pairs only die as the distance grows and the tiles are walked outwards
+// from the diagonal, so the zeroing is monotone).  The MMA depth of a tile is what the nearest
+// quarter keeps, rounded up to a 16-column step.  Coarse mode: depth = pairs live anywhere in the
+// tile rounded up to 8, every pair on the diagonal tile, no per-cell work.  Term counts are those
+// of atf_prefill, bit for bit.
 // Every wait is bounded and reports through the workspace status words.
 #include <cuda.h>
 
@@ -187,18 +189,23 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
   volatile int* abortp = &s_abort;
   unsigned int fail_site = 0;
 
-  // pairs (counted from the low-frequency end) whose window reaches distance z
-  auto pairs_reaching = [&](int z) {
-    int r = 0;
+  // Pairs (counted from the low-frequency end) whose window reaches distance z.  Every role asks for
+  // non-decreasing distances, so each question keeps its own cursor r into the non-decreasing table.
+  auto pairs_reaching = [&](int& r, int z) {
     while (r < H && sW[r] < z) ++r;
     return H - r;
   };
-  // pairs live in some cell / in every cell of the tile at tile distance dt
-  auto p_any_of = [&](int dt) { return pairs_reaching(dt == 0 ? 0 : dt * T - (T - 1)); };
-  auto p_all_of = [&](int dt) { return pairs_reaching(dt * T + T - 1); };
-  // 16-column MMA steps of the S product of that tile
-  auto natoms_of = [&](int dt) { return (MODE != ATF_MODE_EXACT && dt == 0) ? H / 8 : (p_any_of(dt) + 7) / 8; };
-
+  // For the 32 rows of quarter wq against the 128 keys of the tile at tile distance dt: the smallest distance,
+  // the distance from the quarter's middle row to the tile's middle column, the largest distance
+  auto z_any = [](int dt, int wq) { return dt == 0 ? 0 : dt * T + 32 * wq - (T - 1); };
+  auto z_mid = [](int dt, int wq) { return dt == 0 ? 16 * wq + 15 : dt * T + 32 * wq - 48; };
+  auto z_all = [](int dt, int wq) { return dt * T + 32 * wq + 31; };
+  // 16-column MMA steps of the S product of a tile: what the nearest quarter keeps in the MMA (exact: pairs live
+  // in most of its cells), the pairs live anywhere in the tile rounded up to 8 and everything on the diagonal (coarse)
+  auto natoms_of = [&](int& r, int dt) {
+    if (MODE == ATF_MODE_EXACT) return (pairs_reaching(r, z_mid(dt, 0)) + 7) / 8;
+    return dt == 0 ? H / 8 : (pairs_reaching(r, z_any(dt, 0)) + 7) / 8;
+  };
   if (warp == 0) {
     // =============================== TMA producer ===============================
     if (lane == 0) {
@@ -207,10 +214,13 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
         tma_load_3d(sQhi + kb * BLK_BYTES, &tmQhi, bar(S_QFULL), kb * 64, it * T, bhq);
         tma_load_3d(sQlo + kb * BLK_BYTES, &tmQlo, bar(S_QFULL), kb * 64, it * T, bhq);
       }
+      int r_k = 0;
       auto load_k = [&](int t) {
         const int ks = t & 1;
         if (!wait_or_abort(bar(S_KEMPTY + ks), ((t >> 1) & 1) ^ 1, abortp)) return false;
-        const int nkb = max(1, (natoms_of(t) * 16 + 63) / 64);
+        // 64-column K blocks to load: exact mode also reads the pairs it adds per cell
+        const int cols = MODE == ATF_MODE_EXACT ? 2 * pairs_reaching(r_k, z_any(t, 0)) : 16 * natoms_of(r_k, t);
+        const int nkb = max(1, (cols + 63) / 64);
         mbar_expect_tx(bar(S_KFULL + ks), 2 * nkb * BLK_BYTES);
         for (int kb = 0; kb < nkb; ++kb) {
           tma_load_3d(sK + (2 * ks) * SM::TILE + kb * BLK_BYTES, &tmKhi, bar(S_KFULL + ks), kb * 64, (it - t) * T, bhk);
@@ -249,9 +259,10 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
       };
       bool ok = wait_or_abort(bar(S_QFULL), 0, abortp);
       if (!ok) fail_site = 60;
+      int r_n = 0;
       for (int t = 0; t < nt && ok; ++t) {
         const int sb = t & 1;
-        const int natoms = natoms_of(t);
+        const int natoms = natoms_of(r_n, t);
         ok = wait_or_abort(bar(S_KFULL + sb), (t >> 1) & 1, abortp);
         // the softmax warps hold S(t - 2) in registers: its buffer may be written again
         if (ok && t >= 2) ok = wait_or_abort(bar(S_SREAD + sb), ((t >> 1) - 1) & 1, abortp);
@@ -290,13 +301,27 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
     const __nv_bfloat16* qhi_src = P.Qhi + qrow * D;
     const __nv_bfloat16* qlo_src = P.Qlo + qrow * D;
 
+    const int wq = warp & 3;
     bool ok = true;
     int zeroed_from = H;  // pairs p >= zeroed_from are zero in this row of the shared copies of Q
+    auto zero_q_down_to = [&](int p_keep) {
+      for (int p = p_keep; p < zeroed_from; ++p) {
+        const int col = 2 * p;
+        const uint32_t off = (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) + (col & 7) * 2;
+        *reinterpret_cast<uint32_t*>(smem_gen + SM::QHI_OFF + off) = 0u;
+        *reinterpret_cast<uint32_t*>(smem_gen + SM::QLO_OFF + off) = 0u;
+      }
+      zeroed_from = min(zeroed_from, p_keep);
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(S_QZ));
+    };
+    int r_any = 0, r_mid = 0, r_all = 0, r_n = 0;
+    int p_mid = pairs_reaching(r_mid, z_mid(0, wq));  // of the step at hand; the next one's is taken a step ahead
     if (MODE == ATF_MODE_EXACT) {
       ok = wait_or_abort(bar(S_QFULL), 0, abortp);
       if (!ok) fail_site = 70;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(S_QZ));  // step 0: every pair is live on the diagonal
+      if (ok) zero_q_down_to(p_mid);
     }
     float m_used = -INFINITY, l_run = 0.f;  // m_used in raw score units
     unsigned long long cnt = 0;
@@ -304,67 +329,81 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
     for (int t = 0; t < nt && ok; ++t) {
       const int sb = t & 1;
       const int dt = t;
-      const int p_any = p_any_of(dt), p_all = p_all_of(dt);
+      const int p_any = pairs_reaching(r_any, z_any(dt, wq)), p_all = pairs_reaching(r_all, z_all(dt, wq));
+      const int natoms = natoms_of(r_n, dt);
+      const int p_mid_next = t + 1 < nt ? pairs_reaching(r_mid, z_mid(dt + 1, wq)) : 0;
       const int zrow = dt * T + row;  // distance from this row to column 0 of the key tile
       const uint32_t tS = tmem_base + sb * T + lane_off;
       const uint32_t tP = tmem_base + 3 * T + sb * 64 + lane_off;
       if (!wait_or_abort(bar(S_SFULL + sb), (t >> 1) & 1, abortp)) { ok = false; fail_site = 71; break; }
       tc_fence_after();
-      if (MODE == ATF_MODE_EXACT && t + 1 < nt) {
-        // S(t) is complete, so Q is not being read: zero what is live nowhere in the next tile
-        const int p_keep = p_any_of(dt + 1);
-        for (int p = p_keep; p < zeroed_from; ++p) {
-          const int col = 2 * p;
-          const uint32_t off = (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) + (col & 7) * 2;
-          *reinterpret_cast<uint32_t*>(smem_gen + SM::QHI_OFF + off) = 0u;
-          *reinterpret_cast<uint32_t*>(smem_gen + SM::QLO_OFF + off) = 0u;
-        }
-        zeroed_from = min(zeroed_from, p_keep);
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(S_QZ));
-      }
+      // S(t) is complete, so Q is not being read: zero what the quarter does not keep in the MMA of the next tile
+      if (MODE == ATF_MODE_EXACT && t + 1 < nt) zero_q_down_to(p_mid_next);
       float s[T];
+      if (natoms > 0) {
 #pragma unroll
-      for (int q4 = 0; q4 < T / 32; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-      tc_wait_ld();
+        for (int q4 = 0; q4 < T / 32; ++q4) tc_ld32(tS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+        tc_wait_ld();
+      } else {  // no pair is kept in the MMA of this tile: nothing was written, every live term is added below
+#pragma unroll
+        for (int c = 0; c < T; ++c) s[c] = 0.f;
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(S_SREAD + sb));
 
-      // ---- straddling pairs [p_all, p_any): in the MMA depth; take their term back out of the
-      //      cells beyond the pair's window (columns c < zrow - w), 32 columns at a time ----
+      // ---- straddling pairs.  Pairs [p_all, p_mid) went through the MMA: take their three products back
+      //      out of the cells beyond the pair's window.  Pairs [p_mid, p_any) did not (zero in Q): add them in
+      //      the cells inside the window.  32 columns at a time, skipping what no row of the warp needs. ----
       if (MODE == ATF_MODE_EXACT && p_all < p_any) {
         if (!wait_or_abort(bar(S_KFULL + sb), (t >> 1) & 1, abortp)) { ok = false; fail_site = 72; break; }
-        const int zw_hi = dt * T + (warp & 3) * 32 + 31;  // largest zrow of the warp
+        const int zw_lo = dt * T + wq * 32, zw_hi = zw_lo + 31;  // zrow over the warp's rows
         for (int p = p_all; p < p_any; ++p) {
           const int wp = sW[H - 1 - p];
-          const int jb_max = zw_hi - wp;  // columns below it are dead for some row of the warp
-          if (jb_max <= 0) continue;
+          const bool subtract = p < p_mid;
+          // distances of the warp's cells in the chunk of columns 32 q4 .. 32 q4 + 31: [zw_lo - 32 q4 - 31, zw_hi - 32 q4]
+          bool touched[T / 32];
+          bool any = false;
+#pragma unroll
+          for (int q4 = 0; q4 < T / 32; ++q4) {
+            const int hi = zw_hi - 32 * q4, lo = zw_lo - 32 * q4 - 31;
+            touched[q4] = subtract ? (hi > wp) : (lo <= wp && hi >= 0);
+            any |= touched[q4];
+          }
+          if (!any) continue;
           const uint32_t qh = *reinterpret_cast<const uint32_t*>(qhi_src + 2 * p);
           const uint32_t ql = *reinterpret_cast<const uint32_t*>(qlo_src + 2 * p);
-          const float qh0 = bf16lo_to_f32(qh), qh1 = bf16hi_to_f32(qh);
-          const float qs0 = qh0 + bf16lo_to_f32(ql), qs1 = qh1 + bf16hi_to_f32(ql);  // exact: 16 significant bits
+          float qh0 = bf16lo_to_f32(qh), qh1 = bf16hi_to_f32(qh);
+          float qs0 = qh0 + bf16lo_to_f32(ql), qs1 = qh1 + bf16hi_to_f32(ql);  // exact: 16 significant bits
+          if (subtract) {
+            qh0 = -qh0; qh1 = -qh1; qs0 = -qs0; qs1 = -qs1;
+          }
           const int col = 2 * p;
           const uint32_t khi = sK + (2 * sb) * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
           const int chunk = (col & 63) >> 3;
+          // cells with column >= jb = zrow - w are inside the window: adding uses sat(c - jb + 1), taking back sat(jb - c)
           const float jbf = (float)(zrow - wp);
+          const float ca = subtract ? -1.f : 1.f, cb = subtract ? jbf : 1.f - jbf;
 #pragma unroll
           for (int q4 = 0; q4 < T / 32; ++q4) {
-            if (32 * q4 < jb_max) {  // warp-uniform
+            if (touched[q4]) {  // warp-uniform
+              uint32_t kh[32], kl[32];
 #pragma unroll
               for (int cc = 0; cc < 32; ++cc) {
                 const int c = 32 * q4 + cc;
                 const uint32_t a = khi + ((chunk ^ (c & 7)) << 4) + c * 128;
-                uint32_t kh, kl;
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kh) : "r"(a));
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kl) : "r"(a + SM::TILE));
-                float term = qs0 * bf16lo_to_f32(kh);
-                term = fmaf(qs1, bf16hi_to_f32(kh), term);
-                term = fmaf(qh0, bf16lo_to_f32(kl), term);
-                term = fmaf(qh1, bf16hi_to_f32(kl), term);
-                const float dead = __saturatef(jbf - (float)c);  // 1 for c < zrow - w, else 0
-                s[c] = fmaf(-term, dead, s[c]);
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kh[cc]) : "r"(a));
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kl[cc]) : "r"(a + SM::TILE));
+              }
+#pragma unroll
+              for (int cc = 0; cc < 32; ++cc) {
+                const int c = 32 * q4 + cc;
+                float term = qs0 * bf16lo_to_f32(kh[cc]);
+                term = fmaf(qs1, bf16hi_to_f32(kh[cc]), term);
+                term = fmaf(qh0, bf16lo_to_f32(kl[cc]), term);
+                term = fmaf(qh1, bf16hi_to_f32(kl[cc]), term);
+                const float coef = __saturatef(fmaf(ca, (float)c, cb));
+                s[c] = fmaf(term, coef, s[c]);
               }
             }
           }
@@ -389,7 +428,7 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
             cnt += (unsigned long long)max(0, hi - lo + 1);
           }
         } else {
-          cnt += (unsigned long long)min(H, 8 * natoms_of(dt)) * (unsigned long long)ncols;
+          cnt += (unsigned long long)min(H, 8 * natoms) * (unsigned long long)ncols;
         }
       }
       // ---- online softmax, lazy rescaling ----
@@ -445,6 +484,7 @@ atf_prefill_split_kernel(const __grid_constant__ CUtensorMap tmQhi, const __grid
         mbar_arrive(bar(S_PFULL + sb));
         mbar_arrive(bar(S_KEMPTY + sb));
       }
+      p_mid = p_mid_next;
     }
     if (ok && nt > 0) {
       if (!wait_or_abort(bar(S_OFULL), 0, abortp)) {
