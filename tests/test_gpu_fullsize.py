@@ -161,3 +161,58 @@ def test_qwen7b_1m_prefill_counts_and_rows(atf):
         o, l = orc._softmax_row(s, Vr[: n + 1])
         _check_rows(gen.to_f64(O[0, hq, n])[None, :], o[None, :], n)
         assert abs(float(LSE[0, hq, n]) - l) <= LSE_TOL
+
+
+@pytest.mark.parametrize("B,L", [(1, 131072), (8, 32768)])
+def test_llama_decode_unrotated_cache_fullsize(atf, B, L):
+    """The benchmark's decode shapes on an unrotated group-major cache (rotation at read, App. B): the oracle
+    rotates the stored keys itself and decodes; three (batch, head) samples and every head's term count."""
+    w = gen.llama32_3b(L, B=B, seed_off=27 + (B > 1))
+    q, Ku, Vc = gen.decode_inputs(w, device="cuda")     # Ku: keys before RoPE
+    W, theta = atf.atf_window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Wo, theta_o = orc.window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Kg = atf.atf_kcache_pack(Ku)
+    tabs = atf.atf_rope_tables(theta, w.d, L)
+    kept = torch.zeros(w.B * w.Hq, dtype=torch.int64, device="cuda")
+    O, lse = atf.atf_decode(q, Kg, Vc, table=W, kept_terms=kept, return_lse=True, rope_tables=tabs)
+    torch.cuda.synchronize()
+    atf.binding.check_status()
+    assert kept.cpu().tolist() == [orc.kept_terms_decode(Wo, L)] * (w.B * w.Hq)
+    g = w.Hq // w.Hkv
+    for b, hq in ((0, 0), (B - 1, 23), (B // 2, 10)):
+        Kr = orc.rope_half_split(gen.to_f64(Ku[b:b + 1, hq // g:hq // g + 1]), theta_o)
+        Or, Lr = orc.decode(gen.to_f64(q[b:b + 1, hq:hq + 1]), Kr, gen.to_f64(Vc[b:b + 1, hq // g:hq // g + 1]), Wo)
+        err = np.abs(gen.to_f64(O[b, hq]) - Or[0, 0])
+        assert err.max() <= O_MAX and err.mean() <= O_MEAN
+        assert abs(float(lse[b, hq]) - Lr[0, 0]) <= LSE_TOL
+
+
+def test_llama_32768_split_precision(atf):
+    """Split-precision prefill at the 32K Llama shape (whole problem on the GPU), sampled rows of two heads
+    against the definition on the fp32 values, every head's term count."""
+    w = gen.llama32_3b(32768, seed_off=31)
+    Q, K, V = gen.prefill_inputs_f32(w, device="cuda")
+    W, theta = atf.atf_window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Wo, theta_o = orc.window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Qg, Kg = Q.clone(), K.clone()
+    atf.atf_rope_f32(Qg, theta)
+    atf.atf_rope_f32(Kg, theta)
+    kept = torch.zeros(w.B * w.Hq, dtype=torch.int64, device="cuda")
+    O, LSE = atf.atf_prefill_split(Qg, Kg, V, table=W, kept_terms=kept)
+    torch.cuda.synchronize()
+    atf.binding.check_status()
+    assert kept.cpu().tolist() == [orc.kept_terms_prefill(Wo, w.N)] * (w.B * w.Hq)
+    rows = gen.sample_rows(w.N, Wo, 24, 91, tile=32)
+    g = w.Hq // w.Hkv
+    for hq in (5, 22):
+        Kr = orc.rope_half_split(K[0, hq // g].cpu().numpy().astype(np.float64), theta_o, 0, round_bf16=False)
+        Kr = Kr.astype(np.float32).astype(np.float64)
+        Qr = np.zeros_like(Kr)
+        qsel = Q[0, hq][rows].cpu().numpy().astype(np.float64)
+        for i, n in enumerate(rows):
+            Qr[n] = orc.rope_half_split(qsel[i:i + 1], theta_o, pos0=n, round_bf16=False)[0].astype(np.float32)
+        Or, Lr = orc.attention_rows(Qr, Kr, gen.to_f64(V[0, hq // g]), Wo, rows)
+        _check_rows(gen.to_f64(O[0, hq])[rows], Or, f"split head {hq}")
+        le = np.abs(LSE[0, hq].double().cpu().numpy()[rows] - Lr)
+        smax = max(np.abs(s[np.isfinite(s)]).max() for s in (orc.windowed_scores_row(Qr[n], Kr, Wo, n) for n in rows[::16]))
+        assert le.max() <= 1.5e-5 * max(1.0, smax), (hq, le.max(), smax)
