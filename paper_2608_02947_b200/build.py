@@ -18,8 +18,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libatflash.so")
-SOURCES = ["atf_host.cu", "atf_rope.cu", "atf_decode.cu", "atf_prefill.cu", "atf_prefill_host.cu", "atf_prefill_split.cu"]
-HEADERS = [os.path.join(CSRC, "atf_common.cuh"), os.path.join(ROOT, "include", "atflash.h")]
+SOURCES = ["atf_host.cu", "atf_rope.cu", "atf_decode.cu", "atf_prefill.cu", "atf_prefill_host.cu", "atf_prefill_split.cu", "atf_prefill_pipe.cu"]
+HEADERS = [os.path.join(CSRC, "atf_common.cuh"), os.path.join(CSRC, "atf_prefill_pipe.cuh"), os.path.join(ROOT, "include", "atflash.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 EXTRA = os.environ.get("ATF_NVCC_EXTRA", "").split()
 FLAGS = EXTRA + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -41,7 +41,10 @@
 // every role of the main kernel reads its word one step ahead and does no schedule arithmetic.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "atf_common.cuh"
+#include "atf_prefill_pipe.cuh"
 
 namespace {
 
@@ -947,7 +950,7 @@ atf_status atf_validate_table(const char* who, const int64_t* table, int d, int6
 
 // band schedule: one 16-byte record per tile distance a launch over N keys can meet
 static int sched_entries(int64_t N) { return 2 * (int)((N + 2 * T - 1) / (2 * T)) + 1; }
-static size_t sched_bytes(int64_t N) { return ((size_t)sched_entries(N) * 16 + 255) & ~(size_t)255; }
+static size_t sched_bytes(int64_t N) { return ((size_t)sched_entries(N) * 32 + 255) & ~(size_t)255; }  // room for either pipeline's records
 
 size_t atf_prefill_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int d) {
   return ATF_WS_HEADER + sched_bytes(N) + repack_bytes(B, Hq, N, d) + repack_bytes(B, Hkv, N, d);
@@ -1021,6 +1024,23 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
   if ((st = atf_make_tile_map(&tk, Kp, (int64_t)B * Hkv, N, d, N, T)) != ATF_OK) return st;
   if ((st = atf_make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, kv_head_rows, T)) != ATF_OK) return st;
 
+  {
+    static const int pipe = [] { const char* e = getenv("ATF_PREFILL_PIPE"); return e ? atoi(e) : 1; }();
+    if (pipe) {
+      AtfPipeParams PP;
+      PP.sched = sched;
+      PP.Qp = Qp;
+      PP.O = (__nv_bfloat16*)O;
+      PP.LSE = LSE;
+      PP.kept = opts ? (unsigned long long*)opts->kept_terms : nullptr;
+      PP.status = (unsigned int*)base;
+      PP.Hq = Hq;
+      PP.Hkv = Hkv;
+      PP.N = (int)N;
+      PP.Nq = (int)Nq;
+      return atf_launch_prefill_pipe(tq, tk, tv, PP, t, B, d, mode, PP.kept != nullptr, s);
+    }
+  }
   PrefillParams P;
   P.sched = sched;
   P.Qp = Qp;
