@@ -1,13 +1,14 @@
-// atf_prefill, second pipeline: ONE 128-row query tile per CTA (Sec. 3.3, Fig. 3 on sm_100a).
+// atf_prefill kernel: windowed causal attention for all query rows (Sec. 3.3, Fig. 3) on the sm_100a
+// tensor cores, ONE 128-row query tile of one head per CTA.  (Layout of the operands: atf_prefill.cu.)
 //
-// With a single query tile the 512 tensor-memory columns hold two S buffers, two P buffers and O,
-// so the chain "softmax -> O += P V -> next S -> softmax" of the two-tile kernel is cut: S(t + 1)
-// is computed while the softmax groups work on S(t), and O += P(t) V runs whenever P(t) is
-// stored.  Warp roles:
+// With a single query tile the 512 tensor-memory columns hold two S buffers, two P buffers and O, so
+// the chain "softmax -> O += P V -> next S -> softmax" is cut: S(t + 1) = Q K(t + 1)^T is computed
+// while the softmax groups work on S(t), and O += P(t) V runs whenever P(t) is stored.  Warp roles:
 //   warp 0      TMA producer: Q (again per pass, see below), K (live 64-column blocks) and V
-//               tiles into three-stage rings;
-//   warp 1      issuer of S(t) = Q K(t)^T over the live depth (one thread);
-//   warp 2      issuer of O += P(t) V(t), half a tile at a time (one thread);
+//               tiles into three-stage rings of 128-byte-swizzled shared memory;
+//   warp 1      issuer of S(t) = Q K(t)^T over the live depth (one thread, tcgen05.mma SS form);
+//   warp 2      issuer of O += P(t) V(t), half a tile at a time (one thread, TS form: P is read from
+//               tensor memory, V through the MN-major descriptor);
 //   warps 4-7   softmax group 0: keys 0..63 of every tile, one query row per thread;
 //   warps 8-11  softmax group 1: keys 64..127 of the same rows.
 // The two threads of a row never meet in the common step: exponentials are taken against the
@@ -16,13 +17,23 @@
 // partial row sum, and the halves are added at the end.  A thread whose sum of a step is not
 // below 2^64 raises a flag; the CTA then runs its tile a second time in the safe form (the two
 // groups exchange their row maxima through shared memory every step and rescale O at once).
-// Layout, window rule, exact / coarse modes, term counts and appended rows are those of the
-// two-tile kernel in atf_prefill.cu; the schedule quantities come from per-role cursors into the
-// non-decreasing window table instead of the pre-computed band schedule.
-// Exact mode: whether a pair stays in the MMA is decided per quarter of the rows over the whole
-// 128 keys (the pair is live at the distance from the quarter's middle row to the tile's middle
-// column); a warp then finishes its 32 x 64 cells: pairs in the MMA are taken back out of the
-// cells beyond their window, pairs zeroed in Q are added where live.
+//
+// Steps far from the diagonal and from every window boundary ("plain") need neither the mask nor the
+// per-cell finish and run in a loop of their own, kept small so that it stays in the instruction
+// cache; everything else takes the general step, one step at a time.
+//
+// Exact mode (the per-term definition).  Whether a pair stays in the MMA is decided per quarter of
+// the rows over the whole 128 keys (the pair is live at the distance from the quarter's middle row
+// to the tile's middle column); the pairs a quarter does not keep are zeroed in its rows of the
+// CTA's copy of Q (pairs only die as the distance grows and the tiles are walked outwards from
+// the diagonal, so the zeroing is monotone).  A warp then finishes its 32 x 64 cells on the CUDA
+// cores: pairs in the MMA are taken back out of the cells beyond their window, pairs zeroed in Q
+// are added where live.  Coarse mode: depth = pairs live anywhere in the tile rounded up to 8,
+// everything on the diagonal tile, no per-cell work.
+//
+// Appended rows (App. C, "The interval itself"; Sec. 7.3): the tiles stay aligned at position 0 of the
+// context, the grid covers only the tiles that hold query rows, Q is addressed at tile * 128 - n0.
+// Every wait is bounded and reports through the workspace status words.
 #include <cuda.h>
 
 #include <algorithm>
@@ -119,33 +130,34 @@ struct PipeWord {
 template <int MODE>
 __global__ void __launch_bounds__(128)
 atf_pipe_sched_kernel(const __grid_constant__ AtfTable table, int H, int ndt, uint32_t* __restrict__ out) {
-  const int dt = blockIdx.x * blockDim.x + threadIdx.x;
+  // one thread per word: 16 tile distances x 8 (quarter, half) blocks per CTA, the table in shared memory
+  __shared__ int w[ATF_MAX_PAIRS];
+  if (threadIdx.x < H) w[threadIdx.x] = table.w[threadIdx.x];
+  __syncthreads();
+  const int dt = blockIdx.x * 16 + (threadIdx.x >> 3);
   if (dt >= ndt) return;
-  const int Wmax = table.w[H - 1];
+  const int wq = (threadIdx.x >> 1) & 3, h = threadIdx.x & 1;
+  const int Wmax = w[H - 1];
   auto reaching = [&](int z) {  // pairs (from the low-frequency end) whose window reaches distance z
-    int r = 0;
-    while (r < H && table.w[r] < z) ++r;
-    return H - r;
+    int lo = 0, hi = H;         // first r with w[r] >= z, w non-decreasing
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (w[mid] < z) lo = mid + 1; else hi = mid;
+    }
+    return H - lo;
   };
   const int tile_any = reaching(dt == 0 ? 0 : dt * T - (T - 1));  // live somewhere in the tile
   const int mid0 = reaching(dt == 0 ? 15 : dt * T - 48);           // what the nearest quarter keeps in the MMA
   const int natoms = MODE == ATF_MODE_EXACT ? (mid0 + 7) / 8 : (dt == 0 ? H / 8 : (tile_any + 7) / 8);
   const int cols = MODE == ATF_MODE_EXACT ? 2 * tile_any : 16 * natoms;  // exact mode also reads the pairs it adds per cell
   const int nkb = max(1, (cols + 63) / 64);
-  uint32_t w[8];
-  for (int wq = 0; wq < 4; ++wq)
-    for (int h = 0; h < 2; ++h) {
-      const int zmax = dt * T + 32 * wq + 31 - 64 * h, zmin = dt * T + 32 * wq - 64 * h - 63;
-      const int p_all = reaching(max(0, zmax)), p_any = reaching(max(0, zmin));
-      const int p_mid = reaching(dt == 0 ? 16 * wq + 15 : dt * T + 32 * wq - 48);
-      bool plain = dt > 0 && natoms > 0;
-      if (MODE == ATF_MODE_EXACT) plain = plain && zmax <= Wmax && min(p_all, p_mid) >= max(p_any, p_mid);
-      w[2 * wq + h] = (uint32_t)p_all | ((uint32_t)p_any << 7) | ((uint32_t)p_mid << 14) | ((uint32_t)natoms << 21) |
-                      ((uint32_t)(nkb - 1) << 25) | ((uint32_t)plain << 27);
-    }
-  uint4* o = reinterpret_cast<uint4*>(out + 8 * dt);
-  o[0] = make_uint4(w[0], w[1], w[2], w[3]);
-  o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  const int zmax = dt * T + 32 * wq + 31 - 64 * h, zmin = dt * T + 32 * wq - 64 * h - 63;
+  const int p_all = reaching(max(0, zmax)), p_any = reaching(max(0, zmin));
+  const int p_mid = reaching(dt == 0 ? 16 * wq + 15 : dt * T + 32 * wq - 48);
+  bool plain = dt > 0 && natoms > 0;
+  if (MODE == ATF_MODE_EXACT) plain = plain && zmax <= Wmax && min(p_all, p_mid) >= max(p_any, p_mid);
+  out[8 * dt + 2 * wq + h] = (uint32_t)p_all | ((uint32_t)p_any << 7) | ((uint32_t)p_mid << 14) | ((uint32_t)natoms << 21) |
+                             ((uint32_t)(nkb - 1) << 25) | ((uint32_t)plain << 27);
 }
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -644,9 +656,9 @@ atf_status launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
   const int it0 = (P.N - P.Nq) / T;  // first tile with a query row
   dim3 grid(ntq - it0, P.Hq, B);
   if (mode == ATF_MODE_EXACT)
-    atf_pipe_sched_kernel<ATF_MODE_EXACT><<<(ntq + 127) / 128, 128, 0, s>>>(t, D / 2, ntq, P.sched);
+    atf_pipe_sched_kernel<ATF_MODE_EXACT><<<(ntq + 15) / 16, 128, 0, s>>>(t, D / 2, ntq, P.sched);
   else
-    atf_pipe_sched_kernel<ATF_MODE_COARSE><<<(ntq + 127) / 128, 128, 0, s>>>(t, D / 2, ntq, P.sched);
+    atf_pipe_sched_kernel<ATF_MODE_COARSE><<<(ntq + 15) / 16, 128, 0, s>>>(t, D / 2, ntq, P.sched);
   const int smem = PipeSmem<D>::DYN_BYTES;
 #define ATF_PP_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                 \
