@@ -423,7 +423,7 @@ def run_ours(args):
                      "frac": executed / (pre_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
                      # DRAM bytes of one launch: ncu capture at N = 32768 (511 MB) scaled by N (traffic is the
                      # repacked Q/K, V and O once each, linear in N)
-                     "traffic": 511.1e6 * wl.N / 32768 if wl.name == "llama-3.2-3b" else None,
+                     "traffic": 511.7e6 * wl.N / 32768 if wl.name == "llama-3.2-3b" else None,
                      "kernel": "atf_prefill_pipe_kernel (+ schedule and 2 repack launches, <1% of the time)",
                      "peak_source": f"{pk['source']} sustained bf16 GEMM"},
         "roofline_decode": {"bound": "hbm", "achieved": dbytes / (dec_grp_us * 1e-6) / 1e9, "peak": pk["hbm_gbs"],
