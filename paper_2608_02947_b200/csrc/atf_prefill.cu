@@ -133,6 +133,7 @@ atf_status atf_prefill_impl(const void* Q, const void* K, const void* V, void* O
   AtfPipeParams P;
   P.sched = sched;
   P.Qp = Qp;
+  P.Qp_lo = nullptr;
   P.O = (__nv_bfloat16*)O;
   P.LSE = LSE;
   P.kept = opts ? (unsigned long long*)opts->kept_terms : nullptr;

@@ -46,18 +46,23 @@ namespace {
 constexpr int T = 128;
 constexpr int BLK_BYTES = T * 128;
 constexpr int PP_THREADS = 384;
-constexpr int KS = 3, VS = 3;
 constexpr float RESCALE_THRESHOLD = 8.f;      // safe form: log2 units the reference may lag behind
 constexpr float STALE_REF_GUARD = 1.8446744e19f;  // 2^64: a step's partial row sum must stay below it
 static_assert(128 * 56 + 256 * 224 <= PP_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 
-template <int D>
+// SPLIT (the split-precision mode, atf_prefill_split.cu): Q and K come as bf16 hi and lo parts; the CTA holds both
+// Q parts, a K stage is a hi tile followed by a lo tile, and the rings shrink to two K stages and one V stage.
+template <int D, bool SPLIT>
 struct PipeSmem {
   static constexpr int NB = D / 64;
   static constexpr int TILE = NB * BLK_BYTES;
-  static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = TILE;
-  static constexpr int V_OFF = K_OFF + KS * TILE;
+  static constexpr int QN = SPLIT ? 2 : 1;       // operand parts: hi, lo
+  static constexpr int KS = SPLIT ? 2 : 3;       // ring depths
+  static constexpr int VS = SPLIT ? 1 : 3;
+  static constexpr int KSTAGE = QN * TILE;
+  static constexpr int Q_OFF = 0;                // hi part, then lo part
+  static constexpr int K_OFF = QN * TILE;
+  static constexpr int V_OFF = K_OFF + KS * KSTAGE;
   static constexpr int BAR_OFF = V_OFF + VS * TILE;
   static constexpr int X_OFF = BAR_OFF + 256;  // exchange area of the two softmax groups: [2][128] floats
   static constexpr int TOTAL = X_OFF + 1024;
@@ -90,14 +95,16 @@ __device__ __forceinline__ float ex2_approx(float x) {
 #define ATF_PIPE_POLY_OF_4 1
 #endif
 // P = 2^(s * scale + neg_m) for 64 columns, packed to bf16 pairs, and their fp32 sum; one packed pair in
-// four takes the cubic polynomial on the FMA pipe, the rest MUFU (see atf_prefill.cu).
+// four takes a cubic polynomial on the FMA pipe (relative error < 8e-5, below the bf16 rounding of P), the rest
+// MUFU; POLY = 0 (the split-precision mode, whose row sums must be good to 1e-6) is MUFU only.
+template <int POLY>
 __device__ __forceinline__ float exp_half(float (&s)[64], float scale, float neg_m, uint32_t (&pk)[32]) {
   const float2 sc2 = make_float2(scale, scale), nm2 = make_float2(neg_m, neg_m);
   float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
   for (int c = 0; c < 64; c += 2) {
     float2 x = __ffma2_rn(make_float2(s[c], s[c + 1]), sc2, nm2);
-    if (((c >> 1) & 3) < ATF_PIPE_POLY_OF_4) {
+    if (((c >> 1) & 3) < POLY) {
       x = exp2_poly2(x);
     } else {
       x.x = ex2_approx(x.x);
@@ -175,12 +182,15 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
   }
 }
 
-template <int D, int MODE, bool COUNT>
+template <int D, int MODE, bool COUNT, bool SPLIT>
 __global__ void __launch_bounds__(PP_THREADS, 1)
-atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmQlo,
+                        const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmKlo,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AtfPipeParams P,
                         const __grid_constant__ AtfTable table) {
-  using SM = PipeSmem<D>;
+  using SM = PipeSmem<D, SPLIT>;
+  constexpr int KS = SM::KS, VS = SM::VS;
+  constexpr int POLY = SPLIT ? 0 : ATF_PIPE_POLY_OF_4;
   constexpr int H = D / 2;
   constexpr int NB = D / 64;
   constexpr uint32_t TMEM_COLS = 512;  // S0, S1 (128 each) | O (D) at 256 | P0, P1 (64 each) at 384
@@ -234,6 +244,10 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
+    if (SPLIT) {
+      tma_prefetch_desc(&tmQlo);
+      tma_prefetch_desc(&tmKlo);
+    }
     tma_prefetch_desc(&tmV);
   }
   if (warp == 0) {
@@ -264,21 +278,40 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     for (int pass = 0; pass < 2; ++pass) {
       const int g0 = pass * nt;
       if (lane == 0) {
-        mbar_expect_tx(bar(B_QFULL), SM::TILE);
-        for (int kb = 0; kb < NB; ++kb)
+        mbar_expect_tx(bar(B_QFULL), SM::QN * SM::TILE);
+        for (int kb = 0; kb < NB; ++kb) {
           // rows before n0 do not exist in Q: the (possibly negative) coordinate reads zero fill there
           tma_load_3d(sQ + kb * BLK_BYTES, &tmQ, bar(B_QFULL), kb * 64, it * T - n0, bhq);
-        for (int t = 0; t < nt; ++t) {
-          const int g = g0 + t, ks = g % KS, vs = g % VS;
-          if (!wait_or_abort(bar(B_KEMPTY + ks), ((g / KS) & 1) ^ 1, abortp)) { fail_site = 10; break; }
+          if (SPLIT) tma_load_3d(sQ + SM::TILE + kb * BLK_BYTES, &tmQlo, bar(B_QFULL), kb * 64, it * T - n0, bhq);
+        }
+        auto load_k = [&](int t) {
+          const int g = g0 + t, ks = g % KS;
+          if (!wait_or_abort(bar(B_KEMPTY + ks), ((g / KS) & 1) ^ 1, abortp)) return false;
           const int nkb = PipeWord(__ldg(P.sched + 8 * t)).nkb;
-          mbar_expect_tx(bar(B_KFULL + ks), nkb * BLK_BYTES);
-          for (int kb = 0; kb < nkb; ++kb)
-            tma_load_3d(sK + ks * SM::TILE + kb * BLK_BYTES, &tmK, bar(B_KFULL + ks), kb * 64, (it - t) * T, bhk);
-          if (!wait_or_abort(bar(B_VEMPTY + vs), ((g / VS) & 1) ^ 1, abortp)) { fail_site = 11; break; }
+          mbar_expect_tx(bar(B_KFULL + ks), SM::QN * nkb * BLK_BYTES);
+          for (int kb = 0; kb < nkb; ++kb) {
+            tma_load_3d(sK + ks * SM::KSTAGE + kb * BLK_BYTES, &tmK, bar(B_KFULL + ks), kb * 64, (it - t) * T, bhk);
+            if (SPLIT)
+              tma_load_3d(sK + ks * SM::KSTAGE + SM::TILE + kb * BLK_BYTES, &tmKlo, bar(B_KFULL + ks), kb * 64, (it - t) * T, bhk);
+          }
+          return true;
+        };
+        auto load_v = [&](int t) {
+          const int g = g0 + t, vs = g % VS;
+          if (!wait_or_abort(bar(B_VEMPTY + vs), ((g / VS) & 1) ^ 1, abortp)) return false;
           mbar_expect_tx(bar(B_VFULL + vs), SM::TILE);
           for (int kb = 0; kb < NB; ++kb)
             tma_load_3d(sV + vs * SM::TILE + kb * BLK_BYTES, &tmV, bar(B_VFULL + vs), kb * 64, (it - t) * T, bhk);
+          return true;
+        };
+        if (SPLIT) {
+          // one V stage: V(t) has to wait for O += P(t - 1) V, so K(t + 1) goes first
+          bool pok = nt == 0 || load_k(0);
+          for (int t = 0; t < nt && pok; ++t) pok = (t + 1 >= nt || load_k(t + 1)) && load_v(t);
+          if (!pok) fail_site = 10;
+        } else {
+          for (int t = 0; t < nt; ++t)
+            if (!load_k(t) || !load_v(t)) { fail_site = 10; break; }
         }
       }
       if (!another_pass(pass)) break;
@@ -302,12 +335,16 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
           if (iok && MODE == ATF_MODE_EXACT) iok = wait_or_abort(bar(B_QZ), g & 1, abortp);
           if (!iok) { fail_site = 21; break; }
           tc_fence_after();
-          const uint64_t dK = make_smem_desc_sw128(sK + ks * SM::TILE, 16, 1024);
+          const uint64_t dK = make_smem_desc_sw128(sK + ks * SM::KSTAGE, 16, 1024);
           const uint32_t tS = tmem_base + sb * T;
           for (int a = 0; a < natoms; ++a) {
             // K-major operands advance 32 bytes per 16-column step inside a 64-column block, one block per four steps
             const uint64_t off = (uint64_t)((a & 3) * 2 + (a >> 2) * (BLK_BYTES / 16));
             tc_mma_ss(tS, dQ + off, dK + off, IDESC_QK, a > 0 ? 1u : 0u);
+            if (SPLIT) {  // + Q_hi K_lo^T + Q_lo K_hi^T (the lo parts sit one tile after the hi parts)
+              tc_mma_ss(tS, dQ + off, dK + off + (uint64_t)(SM::TILE / 16), IDESC_QK, 1u);
+              tc_mma_ss(tS, dQ + off + (uint64_t)(SM::TILE / 16), dK + off, IDESC_QK, 1u);
+            }
           }
           tc_commit(bar(B_SFULL + sb));
           if (MODE != ATF_MODE_EXACT) tc_commit(bar(B_KEMPTY + ks));
@@ -360,6 +397,7 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     const uint32_t lane_off = (uint32_t)(wq * 32) << 16;
     const uint32_t tO = tmem_base + 2 * T + lane_off;
     const __nv_bfloat16* qsrc = P.Qp + qrow * D;
+    const __nv_bfloat16* qsrc_lo = SPLIT ? P.Qp_lo + qrow * D : nullptr;
     float m_used = -INFINITY, l_run = 0.f;
     unsigned long long cnt = 0;
     uint32_t xphase = 0;
@@ -385,8 +423,9 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         if (h == 0) {
           for (int p = p_keep; p < zeroed_from; ++p) {
             const int col = 2 * p;
-            *reinterpret_cast<uint32_t*>(smem_gen + SM::Q_OFF + (col >> 6) * BLK_BYTES +
-                                         sw128_offset(row, (col & 63) >> 3) + (col & 7) * 2) = 0u;
+            const uint32_t off = (col >> 6) * BLK_BYTES + sw128_offset(row, (col & 63) >> 3) + (col & 7) * 2;
+            *reinterpret_cast<uint32_t*>(smem_gen + SM::Q_OFF + off) = 0u;
+            if (SPLIT) *reinterpret_cast<uint32_t*>(smem_gen + SM::Q_OFF + SM::TILE + off) = 0u;
           }
           zeroed_from = min(zeroed_from, p_keep);
           fence_proxy_async_smem();
@@ -428,7 +467,7 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
           if (COUNT && row_ok)
             cnt += (unsigned long long)(MODE == ATF_MODE_EXACT ? p_all : min(H, 8 * natoms)) * 64ull;
           uint32_t pk[32];
-          const float lsum = exp_half(s, kScaleLog2, -m_used * kScaleLog2, pk);
+          const float lsum = exp_half<POLY>(s, kScaleLog2, -m_used * kScaleLog2, pk);
           overflow |= !(lsum < STALE_REF_GUARD);
           if (g >= 2 && !wait_or_abort(bar(B_PVDONE + sb), ((g - 2) >> 1) & 1, abortp)) { ok = false; fail_site = 35; break; }
           tc_st32(tmem_base + 3 * T + sb * 64 + 32 * h + lane_off, pk);
@@ -492,14 +531,24 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 touched[q] = subtract ? (hi > wp) : (lo <= wp && hi >= 0);
               }
               if (!touched[0] && !touched[1]) continue;
+              // q0, q1: the pair's two elements of this row (hi parts in the split mode); qs0, qs1: hi + lo there
+              // (exact in fp32: 16 significant bits), so that the term below is the three products of the MMA
               const uint32_t qq = *reinterpret_cast<const uint32_t*>(qsrc + 2 * p);
               float q0 = bf16lo_to_f32(qq), q1 = bf16hi_to_f32(qq);
+              float qs0 = q0, qs1 = q1;
+              if (SPLIT) {
+                const uint32_t ql = *reinterpret_cast<const uint32_t*>(qsrc_lo + 2 * p);
+                qs0 += bf16lo_to_f32(ql);
+                qs1 += bf16hi_to_f32(ql);
+              }
               if (subtract) {
                 q0 = -q0;
                 q1 = -q1;
+                qs0 = -qs0;
+                qs1 = -qs1;
               }
               const int col = 2 * p;
-              const uint32_t kb32 = sK + ks * SM::TILE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
+              const uint32_t kb32 = sK + ks * SM::KSTAGE + (col >> 6) * BLK_BYTES + (col & 7) * 2;
               const int chunk = (col & 63) >> 3;
               // cells with column >= jb = zrow - w are inside the window: adding uses sat(c - jb + 1), taking back
               // sat(jb - c), formed on the FMA pipe
@@ -508,16 +557,19 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 #pragma unroll
               for (int q = 0; q < 2; ++q) {
                 if (touched[q]) {  // warp-uniform
-                  uint32_t kk[32];
+                  uint32_t kk[32], kl[SPLIT ? 32 : 1];
 #pragma unroll
                   for (int cc = 0; cc < 32; ++cc) {
                     const int c = 64 * h + 32 * q + cc;  // key of the tile; (c & 7) does not depend on h
                     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kk[cc]) : "r"(kb32 + ((chunk ^ (c & 7)) << 4) + c * 128));
+                    if (SPLIT)
+                      asm volatile("ld.shared.b32 %0, [%1];" : "=r"(kl[cc]) : "r"(kb32 + SM::TILE + ((chunk ^ (c & 7)) << 4) + c * 128));
                   }
 #pragma unroll
                   for (int cc = 0; cc < 32; ++cc) {
                     const int cl = 32 * q + cc;  // column of this thread's half
-                    const float term = fmaf(q0, bf16lo_to_f32(kk[cc]), q1 * bf16hi_to_f32(kk[cc]));
+                    float term = fmaf(qs0, bf16lo_to_f32(kk[cc]), qs1 * bf16hi_to_f32(kk[cc]));
+                    if (SPLIT) term = fmaf(q0, bf16lo_to_f32(kl[cc]), fmaf(q1, bf16hi_to_f32(kl[cc]), term));
                     const float coef = __saturatef(fmaf(ca, (float)cl, cb));
                     s[cl] = fmaf(term, coef, s[cl]);
                   }
@@ -587,7 +639,7 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
           }
         }
         uint32_t pk[32];
-        const float lsum = exp_half(s, kScaleLog2, m_used == -INFINITY ? 0.f : -m_used * kScaleLog2, pk);
+        const float lsum = exp_half<POLY>(s, kScaleLog2, m_used == -INFINITY ? 0.f : -m_used * kScaleLog2, pk);
         overflow |= !(lsum < STALE_REF_GUARD);
         // the product that read the previous contents of this P buffer must be complete
         if (g >= 2 && !wait_or_abort(bar(B_PVDONE + sb), ((g - 2) >> 1) & 1, abortp)) { ok = false; fail_site = 35; break; }
@@ -649,9 +701,10 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
-template <int D>
-atf_status launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AtfPipeParams& P,
-                       const AtfTable& t, int B, int mode, bool count, cudaStream_t s) {
+template <int D, bool SPLIT>
+atf_status launch_pipe(const CUtensorMap& tq, const CUtensorMap& tql, const CUtensorMap& tk, const CUtensorMap& tkl,
+                       const CUtensorMap& tv, const AtfPipeParams& P, const AtfTable& t, int B, int mode, bool count,
+                       cudaStream_t s) {
   const int ntq = (P.N + T - 1) / T;
   const int it0 = (P.N - P.Nq) / T;  // first tile with a query row
   dim3 grid(ntq - it0, P.Hq, B);
@@ -659,12 +712,12 @@ atf_status launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
     atf_pipe_sched_kernel<ATF_MODE_EXACT><<<(ntq + 15) / 16, 128, 0, s>>>(t, D / 2, ntq, P.sched);
   else
     atf_pipe_sched_kernel<ATF_MODE_COARSE><<<(ntq + 15) / 16, 128, 0, s>>>(t, D / 2, ntq, P.sched);
-  const int smem = PipeSmem<D>::DYN_BYTES;
+  const int smem = PipeSmem<D, SPLIT>::DYN_BYTES;
 #define ATF_PP_LAUNCH(MODE_, COUNT_)                                                                   \
   do {                                                                                                 \
-    auto kern = atf_prefill_pipe_kernel<D, MODE_, COUNT_>;                                             \
+    auto kern = atf_prefill_pipe_kernel<D, MODE_, COUNT_, SPLIT>;                                      \
     ATF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));     \
-    kern<<<grid, PP_THREADS, smem, s>>>(tq, tk, tv, P, t);                                             \
+    kern<<<grid, PP_THREADS, smem, s>>>(tq, tql, tk, tkl, tv, P, t);                                   \
   } while (0)
   if (mode == ATF_MODE_EXACT) {
     if (count) ATF_PP_LAUNCH(ATF_MODE_EXACT, true); else ATF_PP_LAUNCH(ATF_MODE_EXACT, false);
@@ -681,5 +734,13 @@ atf_status launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
 atf_status atf_launch_prefill_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                    const AtfPipeParams& P, const AtfTable& t, int B, int d, int mode, bool count,
                                    cudaStream_t s) {
-  return d == 64 ? launch_pipe<64>(tq, tk, tv, P, t, B, mode, count, s) : launch_pipe<128>(tq, tk, tv, P, t, B, mode, count, s);
+  return d == 64 ? launch_pipe<64, false>(tq, tq, tk, tk, tv, P, t, B, mode, count, s)
+                 : launch_pipe<128, false>(tq, tq, tk, tk, tv, P, t, B, mode, count, s);
+}
+
+atf_status atf_launch_prefill_pipe_split(const CUtensorMap& tqh, const CUtensorMap& tql, const CUtensorMap& tkh,
+                                         const CUtensorMap& tkl, const CUtensorMap& tv, const AtfPipeParams& P,
+                                         const AtfTable& t, int B, int d, int mode, bool count, cudaStream_t s) {
+  return d == 64 ? launch_pipe<64, true>(tqh, tql, tkh, tkl, tv, P, t, B, mode, count, s)
+                 : launch_pipe<128, true>(tqh, tql, tkh, tkl, tv, P, t, B, mode, count, s);
 }
