@@ -47,6 +47,7 @@ constexpr int T = 128;
 constexpr int BLK_BYTES = T * 128;
 constexpr int PP_THREADS = 384;
 constexpr float RESCALE_THRESHOLD = 8.f;      // safe form: log2 units the reference may lag behind
+constexpr float REF_HEADROOM = 60.f;            // fast pass: log2 units the row's reference sits above the diagonal tile's maximum
 constexpr float STALE_REF_GUARD = 1.8446744e19f;  // 2^64: a step's partial row sum must stay below it
 static_assert(128 * 56 + 256 * 224 <= PP_THREADS * 168, "setmaxnreg budget exceeds the launch allocation");
 
@@ -620,6 +621,10 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
           if (mx > m_used && (m_used == -INFINITY || (mx - m_used) * kScaleLog2 > RESCALE_THRESHOLD)) {
             scale_o = m_used == -INFINITY ? 0.f : ex2_approx((m_used - mx) * kScaleLog2);
             m_used = mx;
+            // Fast pass: the reference stays for the whole row, so it is put REF_HEADROOM above the diagonal tile's
+            // maximum: sums overflow only ~120 log2 units above that maximum instead of ~60, and what the shift can
+            // flush to zero lies 2^-66 below the diagonal's own largest term.
+            if (!safe) m_used += REF_HEADROOM / kScaleLog2;
             moved = t > 0;  // nothing has been accumulated before the first tile
           }
           if (__any_sync(0xffffffffu, moved)) {

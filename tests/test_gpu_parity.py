@@ -133,6 +133,19 @@ def test_prefill_tiny_config(atf):
     assert (On.float() - ref).abs().max() <= O_MAX
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_prefill_outlier_logits_take_the_safe_pass(atf, d):
+    """Four pairs scaled by 8 give logits in the hundreds.  The fast path takes every exponential against the
+    row's reference maximum from the diagonal tile; here later keys exceed it by far more than 2^64 for most rows,
+    so a tile's fast pass ends with infinite partial sums and the CTA must run the tile again with the exchanged,
+    running maximum.  Results and term counts must be the definition's all the same (a fast path that went
+    unnoticed would return NaN or infinity)."""
+    w = gen.Workload("outlier", 1, 2, 1, d, 900, 1e4, 2.0, None, gen.SEED0 + 300 + d, True)
+    O, LSE = _prefill_case(atf, w, None, atf.ATF_MODE_EXACT)
+    assert torch.isfinite(LSE).all() and float(LSE.abs().max()) > 60      # the logits really are that large
+    _prefill_case(atf, w, None, atf.ATF_MODE_COARSE)
+
+
 def _decode_case(atf, w: gen.Workload, mode, table=None):
     q, Kc, Vc = gen.decode_inputs(w)
     Wt, _ = atf.atf_window_table(w.base, w.d, w.k, w.N, w.scaling)
