@@ -442,6 +442,7 @@ atf_decode_kernel(const __grid_constant__ DecodeParams P, const __grid_constant_
     float acc[D / 32];
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+#pragma unroll 8
     for (int sp = 0; sp < P.nsplit; ++sp) {
       const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
       const float f = ex2f(__ldcg(src) - Ms);
@@ -851,6 +852,7 @@ atf_decode_tiles_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_co
     float acc[D / 32];
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+#pragma unroll 8
     for (int sp = 0; sp < P.nsplit; ++sp) {
       const float* src = allp + ((int64_t)sp * G + gg) * PSTRIDE;
       const float f = ex2f(__ldcg(src) - Ms);
