@@ -166,6 +166,10 @@ atf_status atf_prefill_ex(const void* Q, const void* K, const void* V, void* O, 
  * ("The interval itself"), whose two end points are the whole prefill and the decode step, and
  * the chunked prefill of Sec. 7.3.  Every row gets exactly what atf_prefill gives it at that
  * position of a length-N prompt, so a prefill cut into chunks has the bits of the single shot.
+ * (One exception, rounding-sized: a 128-row tile whose logits rise more than ~120 log2 units above
+ * its diagonal maximum is recomputed with a running maximum; if a cut falls INSIDE such a tile and the
+ * rows that trigger it lie before the cut, the rows after it differ from the single shot in the last
+ * bit of P.  Cuts at multiples of 128, as atf_prefill_host makes, never do.)
  *   Q, O: dev bf16 [B, Hq, Nq, d];  LSE: dev fp32 [B, Hq, Nq] or NULL;
  *   K, V: dev bf16 [B, Hkv, N, d], rotated at positions 0..N-1;  1 <= Nq <= N (else
  *   ATF_ERR_INVALID_ARG).  table, causal, opts, workspace, errors: as atf_prefill; the table's
@@ -181,7 +185,7 @@ atf_status atf_prefill_chunk_ex(const void* Q, const void* K, const void* V, voi
 
 /* Prefill from and to HOST memory.  Same arguments and results as atf_prefill_ex, but Qh, Kh, Vh,
  * Oh (bf16) and LSEh (fp32 or NULL) are HOST pointers, [B,H,N,d] / [B,Hq,N] dense.  The prompt is
- * processed in chunks of chunk_rows query rows (0 = 16384) as successive appended-rows steps
+ * processed in chunks of chunk_rows query rows (rounded up to a multiple of 128; 0 = 16384) as successive appended-rows steps
  * (see atf_prefill_chunk; bit-identical to the single shot for every chunk size), so that the
  * host->device copy of the next chunk, the kernels of this one and the device->host copy of the
  * previous one overlap on three streams.  Page-locked host buffers are needed for that overlap;

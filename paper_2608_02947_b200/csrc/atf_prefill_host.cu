@@ -31,7 +31,10 @@ struct HostPlan {
 
 HostPlan make_plan(int B, int Hq, int Hkv, int64_t N, int d, int64_t chunk_rows) {
   HostPlan p;
-  p.chunk = std::min<int64_t>(chunk_rows > 0 ? chunk_rows : DEFAULT_CHUNK, N);
+  // chunks start at multiples of the kernel's 128-row tile: a cut inside a tile could change which pass a tile
+  // takes (see atf_prefill_chunk) and with it the last bit of a result
+  const int64_t want = chunk_rows > 0 ? (chunk_rows + 127) / 128 * 128 : DEFAULT_CHUNK;
+  p.chunk = std::min<int64_t>(want, N);
   // workspace of one chunk call: header + repacked Q chunk + repacked K of up to N rows
   p.ws = align256(atf_prefill_workspace_bytes(B, Hq, Hkv, N, d));
   p.kv = align256((size_t)B * Hkv * N * d * 2);
