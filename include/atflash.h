@@ -243,6 +243,11 @@ atf_status atf_decode_ex(const void* q, const void* Kcache, const void* Vcache, 
 atf_status atf_prefill_split(const float* Q, const float* K, const void* V, void* O, float* LSE, int B,
                              int Hq, int Hkv, int64_t N, int d, const int64_t* table, int causal,
                              const atf_opts* opts, void* stream);
+/* The same for Nq rows appended to a context of N keys (Q, O: [B, Hq, Nq, d]; LSE: [B, Hq, Nq]; the rows sit
+ * at positions N-Nq..N-1), as atf_prefill_chunk is to atf_prefill; atf_prefill_split is the Nq = N case. */
+atf_status atf_prefill_split_chunk(const float* Q, const float* K, const void* V, void* O, float* LSE,
+                                   int B, int Hq, int Hkv, int64_t Nq, int64_t N, int d,
+                                   const int64_t* table, int causal, const atf_opts* opts, void* stream);
 atf_status atf_rope_f32(float* X, int B, int H, int64_t N, int d, const double* theta, int64_t pos0,
                         void* stream);
 

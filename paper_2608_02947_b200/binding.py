@@ -57,6 +57,7 @@ def lib():
     L.atf_prefill.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_split.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
     L.atf_rope_f32.argtypes = [vp, i, i, i64, i, C.POINTER(C.c_double), i64, vp]
+    L.atf_prefill_split_chunk.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
     L.atf_prefill_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i, C.POINTER(C.c_int64), i, C.POINTER(_Opts), vp]
     L.atf_prefill_chunk.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i, vp]
     L.atf_prefill_chunk_ex.argtypes = [vp, vp, vp, vp, vp, i, i, i, i64, i64, i, C.POINTER(C.c_int64), i,
@@ -86,7 +87,7 @@ def lib():
     L.atf_last_error.restype = C.c_char_p
     for name in ("atf_window_table", "atf_window_table_family", "atf_rope", "atf_prefill", "atf_prefill_ex", "atf_prefill_chunk",
                  "atf_prefill_chunk_ex", "atf_prefill_host", "atf_decode", "atf_decode_ex",
-                 "atf_kcache_pack", "atf_rope_tables", "atf_prefill_split", "atf_rope_f32",
+                 "atf_kcache_pack", "atf_rope_tables", "atf_prefill_split", "atf_prefill_split_chunk", "atf_rope_f32",
                  "atf_bind_workspace", "atf_check_status", "atf_check_status_at", "atf_selftest_bounded_wait", "atf_probe_masked_read"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -322,27 +323,27 @@ def atf_prefill_split(Q, K, V, table=None, causal=True, mode=ATF_MODE_EXACT, kep
                       O=None, LSE=None):
     """atf_prefill with split-precision scores: Q [B,Hq,N,d] and K [B,Hkv,N,d] are CUDA fp32 (rotated, never
     rounded to bf16), V is bf16; each score is three bf16 tensor-core products (hi*hi + hi*lo + lo*hi).
-    Returns (O bf16, LSE fp32 or None)."""
+    Q may hold only the last Nq rows of the N-key context (appended rows).  Returns (O bf16, LSE fp32 or None)."""
     _dev_f32(Q, "Q")
     _dev_f32(K, "K")
     _dev_bf16(V, "V")
-    B, Hq, N, d = Q.shape
-    Hkv = K.shape[1]
+    B, Hq, Nq, d = Q.shape
+    Hkv, N = K.shape[1], K.shape[2]
     if K.shape != (B, Hkv, N, d) or V.shape != K.shape:
         raise AtfError(1, "K and V must be [B,Hkv,N,d] matching Q")
     if O is None:
         O = torch.empty(Q.shape, dtype=torch.bfloat16, device=Q.device)
     _dev_bf16(O, "O")
     if LSE is None and return_lse:
-        LSE = torch.empty((B, Hq, N), dtype=torch.float32, device=Q.device)
+        LSE = torch.empty((B, Hq, Nq), dtype=torch.float32, device=Q.device)
     dev = _one_device(Q, K, V, O, LSE, kept_terms)
     ensure_workspace(atf_workspace_bytes(ATF_OP_PREFILL_SPLIT, B, Hq, Hkv, N, d), Q.device)
     tab, _keep = _table_ptr(table, d)
     o = _opts(mode, kept_terms, None)
     with dev:
-        _check(lib().atf_prefill_split(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
-                                       C.c_void_p(O.data_ptr()), C.c_void_p(LSE.data_ptr()) if LSE is not None else None,
-                                       B, Hq, Hkv, N, d, tab, 1 if causal else 0,
+        _check(lib().atf_prefill_split_chunk(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                             C.c_void_p(O.data_ptr()), C.c_void_p(LSE.data_ptr()) if LSE is not None else None,
+                                             B, Hq, Hkv, Nq, N, d, tab, 1 if causal else 0,
                                        C.byref(o) if o is not None else None, _stream(Q)))
     return O, LSE
 

@@ -65,12 +65,13 @@ size_t atf_prefill_split_workspace_bytes(int B, int Hq, int Hkv, int64_t N, int 
   return ATF_WS_HEADER + split_sched_bytes(N) + 2 * part_bytes(B, Hq, N, d) + 2 * part_bytes(B, Hkv, N, d);
 }
 
-extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const void* V, void* O, float* LSE, int B, int Hq,
-                                        int Hkv, int64_t N, int d, const int64_t* table, int causal,
-                                        const atf_opts* opts, void* stream) {
+extern "C" atf_status atf_prefill_split_chunk(const float* Q, const float* K, const void* V, void* O, float* LSE, int B,
+                                              int Hq, int Hkv, int64_t Nq, int64_t N, int d, const int64_t* table,
+                                              int causal, const atf_opts* opts, void* stream) {
   if (!Q || !K || !V || !O) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill_split: null pointer");
   if (d != 64 && d != 128) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill_split: d must be 64 or 128 (got %d)", d);
   if (B < 1 || Hq < 1 || Hkv < 1 || N < 1) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill_split: bad shape");
+  if (Nq < 1 || Nq > N) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill_split: need 1 <= Nq <= N (got Nq = %lld, N = %lld)", (long long)Nq, (long long)N);
   if (Hq % Hkv) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill_split: Hq must be a multiple of Hkv");
   if (!causal) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill_split: only causal attention is defined (distance z = n - m >= 0)");
   if (N >= (1ll << 31) - 4 * T) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill_split: N too large");
@@ -93,7 +94,7 @@ extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const vo
   if ((uintptr_t)ws.ptr & 255) return atf_fail(ATF_ERR_INVALID_ARG, "atf_prefill_split: workspace must be 256-byte aligned");
 
   char* base = (char*)ws.ptr;
-  const size_t qb = part_bytes(B, Hq, N, d), kb = part_bytes(B, Hkv, N, d);
+  const size_t qb = part_bytes(B, Hq, Nq, d), kb = part_bytes(B, Hkv, N, d);
   char* parts = base + ATF_WS_HEADER + split_sched_bytes(N);
   __nv_bfloat16* Qhi = (__nv_bfloat16*)parts;
   __nv_bfloat16* Qlo = (__nv_bfloat16*)(parts + qb);
@@ -101,7 +102,7 @@ extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const vo
   __nv_bfloat16* Klo = (__nv_bfloat16*)(parts + 2 * qb + kb);
   cudaStream_t s = (cudaStream_t)stream;
   {
-    const int64_t rows_q = (int64_t)B * Hq * N, rows_k = (int64_t)B * Hkv * N;
+    const int64_t rows_q = (int64_t)B * Hq * Nq, rows_k = (int64_t)B * Hkv * N;
     const int64_t bq = (rows_q * (d / 8) + 255) / 256, bk = (rows_k * (d / 8) + 255) / 256;
     if (bq > 0x7FFFFFFF) return atf_fail(ATF_ERR_UNSUPPORTED, "atf_prefill_split: problem too large for the repack grid");
     atf_split_repack_kernel<<<(unsigned)bq, 256, 0, s>>>(Q, Qhi, Qlo, rows_q, d);
@@ -109,8 +110,8 @@ extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const vo
     ATF_CUDA_CHECK(cudaGetLastError());
   }
   CUtensorMap tqh, tql, tkh, tkl, tv;
-  if ((st = atf_make_tile_map(&tqh, Qhi, (int64_t)B * Hq, N, d, N, T)) != ATF_OK) return st;
-  if ((st = atf_make_tile_map(&tql, Qlo, (int64_t)B * Hq, N, d, N, T)) != ATF_OK) return st;
+  if ((st = atf_make_tile_map(&tqh, Qhi, (int64_t)B * Hq, Nq, d, Nq, T)) != ATF_OK) return st;
+  if ((st = atf_make_tile_map(&tql, Qlo, (int64_t)B * Hq, Nq, d, Nq, T)) != ATF_OK) return st;
   if ((st = atf_make_tile_map(&tkh, Khi, (int64_t)B * Hkv, N, d, N, T)) != ATF_OK) return st;
   if ((st = atf_make_tile_map(&tkl, Klo, (int64_t)B * Hkv, N, d, N, T)) != ATF_OK) return st;
   if ((st = atf_make_tile_map(&tv, V, (int64_t)B * Hkv, N, d, N, T)) != ATF_OK) return st;
@@ -126,6 +127,12 @@ extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const vo
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.N = (int)N;
-  P.Nq = (int)N;
+  P.Nq = (int)Nq;
   return atf_launch_prefill_pipe_split(tqh, tql, tkh, tkl, tv, P, t, B, d, mode, P.kept != nullptr, s);
+}
+
+extern "C" atf_status atf_prefill_split(const float* Q, const float* K, const void* V, void* O, float* LSE, int B, int Hq,
+                                        int Hkv, int64_t N, int d, const int64_t* table, int causal,
+                                        const atf_opts* opts, void* stream) {
+  return atf_prefill_split_chunk(Q, K, V, O, LSE, B, Hq, Hkv, N, N, d, table, causal, opts, stream);
 }

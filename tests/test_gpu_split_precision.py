@@ -132,3 +132,21 @@ def test_split_refusals(atf):
         atf.atf_prefill_split(Q, K, V, causal=False)
     with pytest.raises(atf.AtfError):
         atf.atf_prefill_split(Q, K[:, :, :64].contiguous(), V)
+
+
+def test_split_appended_rows_bit_identical_to_single_shot(atf):
+    """Rows cut off at an aligned and at an unaligned position, computed as appended rows, have the bits of the
+    single shot (both modes)."""
+    w = gen.Workload("split", 2, 4, 2, 128, 1100, 1e4, 2.0, None, gen.SEED0 + 240)
+    Wo, theta = orc.window_table(w.base, w.d, w.k, w.N, w.scaling)
+    Qg, Kg, Vg, *_ = _rotated(atf, w, theta)
+    Wt = torch.from_numpy(Wo)
+    for mode in (0, 1):
+        O, L = atf.atf_prefill_split(Qg, Kg, Vg, table=Wt, mode=mode)
+        for n0 in (512, 333, 1099):
+            kept = torch.zeros(w.B * w.Hq, dtype=torch.int64, device="cuda")
+            Oc, Lc = atf.atf_prefill_split(Qg[:, :, n0:].contiguous(), Kg, Vg, table=Wt, mode=mode, kept_terms=kept)
+            assert torch.equal(Oc, O[:, :, n0:]) and torch.equal(Lc, L[:, :, n0:]), (mode, n0)
+            if mode == 0:
+                assert kept.cpu().tolist() == [orc.kept_terms_interval(Wo, n0, w.N)] * (w.B * w.Hq)
+    atf.binding.check_status()
