@@ -481,7 +481,7 @@ atf_prefill_pipe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
           e_cur = e_next;
         }
         if (t >= nt || !ok) break;
-        // ---- one general step (the cursors give the same answers when asked again) ----
+        // ---- one general step ----
         const int g = g0 + t, sb = g & 1, ks = g % KS;
         const int dt = t;
         const int zrow = dt * T + row;             // distance from this row to column 0 of the key tile
